@@ -1,0 +1,194 @@
+/*
+ * dlfusion.h - C ABI of the fused conv-group executor for NVIDIA B200 (sm_100a).
+ *
+ * A network is a list of layers.  A *plan* cuts the list into contiguous fusion groups and
+ * gives each group a number of SMs: the two outputs of the paper's Algorithm 1
+ * (fusion_partition_index[] and mp_of_fusionblock[]) and the two knobs of its Sec. II-A.2
+ * ("model parallelism" = cores used by an operator or block, and "layer fusion").  A group
+ * runs as one kernel whose intermediate feature maps stay in shared / tensor memory
+ * (Sec. III-B: the output of a fused layer is produced on chip and reused at once); a
+ * group's last layer is written to HBM.  All plans compute the same values: activations
+ * are fp16, arithmetic is fp32, and every layer's result is rounded to fp16 once
+ * (round-to-nearest-even) whether or not it leaves the chip.
+ *
+ * Conventions
+ *   - Every call returns an int status: DLF_OK or a negative DLF_E_* code.  Nothing throws,
+ *     aborts or exits.  dlf_strerror() names a code; dlf_last_cuda_error() returns the last
+ *     CUDA runtime/driver error number seen by the calling thread's most recent failing call.
+ *   - Pointers named *_dev are DEVICE pointers, *_host are HOST pointers; everything else
+ *     (descriptors, plans, out-parameters) is host memory.
+ *   - The caller owns all device memory: input, output, weights, biases and one workspace
+ *     whose size the library reports.  The library allocates no device memory.  Device
+ *     pointers are borrowed: they must stay valid until replaced or the net is destroyed.
+ *   - Tensors are NHWC fp16 (IEEE binary16).  Weights are [cout][kh][kw][cin/groups] fp16
+ *     (a fully connected layer: [cout][cin], cin in NHWC-flatten order).  Biases are fp32.
+ *     Device pointers must be 16-byte aligned (256-byte for the workspace).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Calls on one dlf_net must not overlap in time; different nets are independent.
+ */
+#ifndef DLFUSION_H_
+#define DLFUSION_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    DLF_OK = 0,
+    DLF_E_INVALID_ARG = -1, /* null pointer, non-positive size, bad enum                        */
+    DLF_E_SHAPE = -2,       /* layer list does not type-check (channels, empty output, src)     */
+    DLF_E_PLAN = -3,        /* plan is not a contiguous cover, SM count out of range, or a group
+                               cannot run as one kernel (never silently re-partitioned)         */
+    DLF_E_WORKSPACE = -4,   /* workspace missing, misaligned or too small                       */
+    DLF_E_UNSUPPORTED = -5, /* layer type / parameter combination has no kernel                 */
+    DLF_E_CUDA = -6,        /* a CUDA call failed; see dlf_last_cuda_error()                    */
+    DLF_E_TIMEOUT = -7,     /* a bounded device-side wait gave up (status word set by a kernel)  */
+    DLF_E_STATE = -8        /* call out of order: weights or plan missing                       */
+};
+
+typedef enum { DLF_CONV = 0, DLF_DWCONV = 1, DLF_FC = 2, DLF_MAXPOOL = 3, DLF_GAVGPOOL = 4 } dlf_op;
+typedef enum { DLF_ACT_NONE = 0, DLF_ACT_RELU = 1, DLF_ACT_RELU6 = 2 } dlf_act;
+
+/* One layer, in the paper's {C_in, C_out, H_out x W_out, K_h x K_w} notation (Sec. II-B) plus
+ * what the fused epilogue needs.  BatchNorm is folded into the bias. */
+typedef struct {
+    int32_t op;      /* dlf_op                                                                  */
+    int32_t act;     /* dlf_act, applied after bias (and residual)                              */
+    int32_t cin, cout;
+    int32_t kh, kw, stride, pad;
+    int32_t groups;  /* 1 = dense; cin for depthwise (DLF_DWCONV requires groups == cin == cout) */
+    int32_t src;     /* index of the layer whose output this layer reads; -1 = network input    */
+    int32_t res_src; /* -2 = none; -1 = network input; else layer index added before the act.   */
+    int32_t pool;    /* 0, or 2 = 2x2 stride-2 max-pool fused after the activation              */
+} dlf_layer_desc;
+
+/* Parameters of Eq. 5 and Algorithm 1.  Eq. 5 gives a proportionality only, so the per-layer SM
+ * count is clamp(round(kappa * (alpha*log2(C_out) + beta*log2(ops)) + kappa0), 1, s_max), with
+ * ops = Eq. 1 / Eq. 2 times the batch and divided by the groups.  op_critical is Algorithm 1's
+ * OpCount_critical in the same unit (operations per SM). */
+typedef struct {
+    double alpha, beta;   /* paper's MLU100 values: 0.316, 0.659                                 */
+    double kappa, kappa0; /* affine map from the Eq. 5 score to an SM count                      */
+    double op_critical;   /* close a block when sum_ops / avg_sm >= op_critical                  */
+    int32_t s_max;        /* largest SM count (<= SMs of the device); 0 = all SMs                */
+    int32_t legalise;     /* 0: pure Algorithm 1 (blocks close only where no kernel could ever
+                             fuse across: structural rule).  1: also split blocks the fused
+                             kernel cannot hold (shared / tensor memory capacity)                */
+} dlf_tuner_params;
+
+/* Reduced brute-force search (paper Sec. V, "Oracle Case"): every candidate group (a legal span
+ * of at most max_group_len layers, one SM count out of sm_choices) is timed once on the device
+ * and the best contiguous partition is found by dynamic programming over the measured times. */
+typedef struct {
+    int32_t n_sm_choices;
+    int32_t sm_choices[16];
+    int32_t max_group_len;
+    int32_t warmup, iters;
+} dlf_search_params;
+
+typedef struct dlf_net dlf_net;
+
+const char* dlf_strerror(int status);
+int dlf_last_cuda_error(void);
+/* Number of SMs of the current device (the upper limit of the SM-count knob), or a DLF_E_* code. */
+int dlf_device_sm_count(void);
+
+/* Builds a net from n_layers descriptors (copied) for an N x H x W x C fp16 NHWC input.
+ * Infers every layer's output shape, H_out = floor((H + 2 pad - k) / stride) + 1, and its
+ * operation count (Eq. 1 / Eq. 2).  Errors: DLF_E_INVALID_ARG, DLF_E_SHAPE, DLF_E_UNSUPPORTED. */
+int dlf_net_create(const dlf_layer_desc* layers, int n_layers, int N, int H, int W, int C,
+                   dlf_net** out);
+void dlf_net_destroy(dlf_net* net);
+
+/* ops_eq1: Eq. 1 / Eq. 2 exactly as printed (no batch, no groups; this is what reproduces the
+ * paper's Table 2).  flops: useful operations of one run (batch included, divided by groups).
+ * out_shape: {N, H, W, C}.  Any out-pointer may be NULL. */
+int dlf_net_layer_info(const dlf_net* net, int layer, int64_t* ops_eq1, int64_t* flops,
+                       int64_t out_shape[4]);
+
+/* Device pointers to one layer's weights and bias (borrowed).  Layers without parameters
+ * (pools) take none.  Changing weights invalidates nothing else. */
+int dlf_net_set_weights(dlf_net* net, int layer, const void* w_f16_dev, const float* bias_dev);
+
+/* Workspace: staging for the input of dlf_net_run_host, one slot per layer output (the worst
+ * case over plans is the unfused plan, where every layer reaches HBM), scratch for split
+ * reductions and a status word.  Contents are undefined between runs. */
+int dlf_net_workspace_bytes(const dlf_net* net, size_t* bytes);
+int dlf_net_bind_workspace(dlf_net* net, void* workspace_dev, size_t bytes);
+
+/* Sets the plan: group g covers layers (group_end[g-1], group_end[g]] (inclusive end index) and
+ * runs on sm_count[g] SMs (a persistent grid of that many CTAs).  DLF_E_PLAN if the ends are not
+ * strictly increasing up to n_layers-1, an SM count is outside [1, #SMs], or a group with more
+ * than one layer is not a chain the fused kernel can hold. */
+int dlf_net_set_plan(dlf_net* net, int n_groups, const int32_t* group_end, const int32_t* sm_count);
+/* The no-fusion plan: one group per layer, all SMs. */
+int dlf_net_plan_unfused(dlf_net* net);
+/* Reads back the current plan; arrays must hold n_layers entries. */
+int dlf_net_get_plan(const dlf_net* net, int* n_groups, int32_t* group_end, int32_t* sm_count);
+/* 1 if layers first..last can run as one fused kernel on `sm_count` SMs, 0 if not. */
+int dlf_net_group_is_legal(const dlf_net* net, int first, int last, int sm_count);
+
+/* Algorithm 1 with Eq. 5 (host only, O(n)).  Writes the plan into the arrays (n_layers entries
+ * each) and does NOT install it; pass it to dlf_net_set_plan. */
+int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_groups,
+                     int32_t* group_end, int32_t* sm_count);
+
+/* Reduced brute-force search; needs weights and workspace.  Installs nothing; leaves the net's
+ * plan as it was.  best_ms: the dynamic programme's optimum (sum of group times). */
+int dlf_net_bruteforce(dlf_net* net, const dlf_search_params* params, const void* in_dev,
+                       void* stream, int* n_groups, int32_t* group_end, int32_t* sm_count,
+                       float* best_ms);
+
+/* Enqueues one inference on `stream` and returns without waiting.  in_dev: N*H*W*C fp16.
+ * out_dev: the last layer's output, fp16 NHWC.  DLF_E_STATE without weights / plan /
+ * workspace. */
+int dlf_net_run(dlf_net* net, const void* in_f16_dev, void* out_f16_dev, void* stream);
+/* Same with HOST buffers: copies the input to the device, runs, copies the output back and
+ * waits for the stream.  For asynchronous copies the host buffers should be page-locked. */
+int dlf_net_run_host(dlf_net* net, const void* in_f16_host, void* out_f16_host, void* stream);
+/* Waits for the stream and reports a device-side bounded wait that gave up (DLF_E_TIMEOUT)
+ * or a CUDA error from the kernels enqueued so far. */
+int dlf_net_sync(dlf_net* net, void* stream);
+
+/* Times `iters` runs with CUDA events on `stream` after `warmup` untimed ones.  If flush_dev is
+ * non-NULL its flush_bytes are overwritten before every run, outside the timed interval, to
+ * evict L2.  ms_median / ms_min: per-run times.  ms_per_group (may be NULL): median time of
+ * each group from a second, instrumented pass with an event after every group. */
+int dlf_net_time(dlf_net* net, const void* in_dev, void* out_dev, void* stream, int warmup,
+                 int iters, void* flush_dev, size_t flush_bytes, float* ms_median, float* ms_min,
+                 float* ms_per_group);
+
+/* Device pointer and shape of a layer output that the current plan writes to HBM (a group's
+ * last layer); valid after a run.  DLF_E_PLAN for a layer inside a group. */
+int dlf_net_boundary_tensor(const dlf_net* net, int layer, const void** dev_ptr, int64_t shape[4]);
+
+/* Roofline model of group g of the current plan: useful flops, compulsory HBM bytes (the
+ * group's external inputs once, its output, its weights and biases once; maps inside the group
+ * count zero, Eq. 3 applied to the group), the ratio computed/useful multiply-accumulates
+ * including the recomputed halo of the chosen tiling (Sec. IV-B), and the number of kernels the
+ * group launches. */
+int dlf_net_group_model(const dlf_net* net, int group, int64_t* flops, int64_t* hbm_bytes,
+                        double* redundancy, int* launches);
+
+/* Name of the kernel variant that runs group g ("chain_tc", "conv_tc", "conv_direct", "dw3x3",
+ * "fc", "maxpool", "gavgpool"); the string is owned by the library. */
+const char* dlf_net_group_kernel(const dlf_net* net, int group);
+
+/* Options (debugging and ablation); setting one clears the plan, which must be set again.
+ *   DLF_OPT_NO_TENSOR_CORE   1: route every dense convolution to the CUDA-core direct kernel
+ *                               (multi-layer groups then become illegal).
+ *   DLF_OPT_DESC_BASE_OFFSET 1 (default): the fused kernel's shifted shared-memory descriptors
+ *                               carry the row phase of their start address; 0: leave it zero.
+ *   DLF_OPT_SINGLE_AS_CHAIN  1: a single stride-1 1x1 / 3x3 convolution with <= 256 output
+ *                               channels runs through the fused-chain kernel (input tile
+ *                               loaded once) instead of the per-tap kernel. */
+enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3 };
+int dlf_net_set_option(dlf_net* net, int option, int value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DLFUSION_H_ */

@@ -1,0 +1,77 @@
+// Internal declarations shared by the host model, the launcher and the kernels' host wrappers.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/dlfusion.h"
+
+namespace dlf {
+
+// One convolution-like layer as a kernel sees it.  Ho, Wo are the sizes BEFORE a fused pool.
+struct ConvArgs {
+    const void* x;
+    const void* w;
+    const float* bias;
+    const void* res;  // nullable, shape [N][Ho][Wo][Cout]
+    void* y;          // [N][Ho][Wo][Cout], or [N][Ho/2][Wo/2][Cout] with pool == 2
+    int N, H, W, Cin, Ho, Wo, Cout;
+    int kh, kw, stride, pad, groups, act, pool;
+};
+
+// A chain of stride-1, size-keeping dense convolutions executed by one kernel.
+constexpr int kMaxChain = 8;
+struct ChainArgs {
+    int n_layers;
+    const void* x;
+    const void* w[kMaxChain];
+    const float* bias[kMaxChain];
+    int cin[kMaxChain], cout[kMaxChain], k[kMaxChain], act[kMaxChain];
+    const void* res;  // residual added at the last layer, [N][H][W][Cout_last], nullable
+    void* y;
+    int N, H, W;
+    int pool;  // 0 / 2 on the last layer
+};
+
+// Tiling of a chain chosen from the SM-count knob (Sec. IV-B: more cores -> smaller tiles ->
+// more recomputed halo).
+struct ChainTiling {
+    int th, tw;          // output tile of the last layer (before pooling)
+    int halo;            // sum of the layers' paddings
+    int pitch, rows;     // frame of the input tile: (th + 2 halo) x (tw + 2 halo), pitch = width
+    int tiles_h, tiles_w, n_tiles;
+    int stages;          // weight ring depth
+    size_t smem_bytes;
+    int tmem_cols;
+    double redundancy;   // computed / useful multiply-accumulates
+    bool ok;
+};
+
+int cuda_fail(cudaError_t e);  // records the error for dlf_last_cuda_error, returns DLF_E_CUDA
+int cuda_fail_drv(int e);
+
+// kernels_mem.cu
+int launch_conv_direct(const ConvArgs& a, int sm_count, cudaStream_t s);
+int launch_dw3x3(const ConvArgs& a, int sm_count, cudaStream_t s);
+int launch_maxpool(const void* x, void* y, int N, int H, int W, int C, int k, int stride, int pad, int Ho, int Wo,
+                   int sm_count, cudaStream_t s);
+int launch_gavgpool(const void* x, void* y, int N, int H, int W, int C, int sm_count, cudaStream_t s);
+int launch_fc(const void* x, const void* w, const float* bias, void* y, int N, int K, int M, int act, int sm_count,
+              cudaStream_t s);
+
+// conv_tc.cu
+bool conv_tc_supported(const ConvArgs& a);
+int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s);
+
+// chain_tc.cu
+ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms);
+int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int base_offset_mode, int* status_dev,
+                    cudaStream_t s);
+
+// tensor map encoding through the driver entry point (no link-time dependency on libcuda)
+int encode_tmap(void* out_map /*CUtensorMap*/, const void* base, int rank, const uint64_t* dims,
+                const uint64_t* strides_bytes /*rank-1*/, const uint32_t* box, const uint32_t* elem_strides);
+
+}  // namespace dlf

@@ -1,0 +1,154 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU checker, element by element, on
+the same seeded inputs, at every group boundary, under several fusion plans and SM counts."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+from oracle import executor as orc
+from paper_2011_05630_b200 import binding as B, networks as nw, synth
+from paper_2011_05630_b200.runtime import Session
+from tests import gpu_util as G
+from tests.test_oracle_layers import _tiny_resnet_like
+
+
+def _mk(layers, tag, n, h, w, c):
+    params = synth.layer_params(tag, layers)
+    x = synth.network_input(tag, n, h, w, c)
+    ref = orc.run_network(layers, params, x)
+    sess = Session(layers, params, n, h, w, c)
+    return sess, sess.upload(x), ref
+
+
+def _conv(cin, cout, k, stride=1, pad=None, act="relu", pool=0, groups=1, op="conv", src=-1, res_src=-2):
+    return dict(op=op, act=act, cin=cin, cout=cout, kh=k, kw=k, stride=stride, pad=k // 2 if pad is None else pad,
+                groups=groups, src=src, res_src=res_src, pool=pool)
+
+
+SMS = None
+
+
+def sms():
+    global SMS
+    if SMS is None:
+        SMS = B.device_sm_count()
+    return SMS
+
+
+# ---- config 1: the two-layer fusion group -------------------------------------------------------------
+@pytest.mark.parametrize("s", [1, 4, 0])
+def test_two_layer_group_unfused_and_fused(s):
+    s = s or sms()
+    sess, xd, ref = _mk(nw.two_layer_group(), "cfg1", 1, 32, 32, 16)
+    G.check_plan(sess, xd, ref, [0, 1], [s, s], "cfg1 unfused")
+    assert sess.kernels() == ["conv_tc", "conv_tc"]
+    G.check_plan(sess, xd, ref, [1], [s], "cfg1 fused")
+    assert sess.kernels() == ["chain_tc"]
+    # plan invariance on the device itself: fused and unfused agree to rounding flips
+    fused = sess.boundary(1).copy()
+    sess.set_plan([0, 1], [s, s])
+    sess.run(xd)
+    assert G.rel_l2(fused, sess.boundary(1)) < 2e-3
+
+
+# ---- single layers: every kernel variant ------------------------------------------------------------------
+SINGLE = [
+    # (n, h, w, layer)
+    (1, 32, 32, _conv(16, 16, 3)),
+    (2, 19, 23, _conv(64, 64, 3)),                 # ragged tiles
+    (1, 56, 56, _conv(64, 128, 1, act="none")),
+    (3, 14, 14, _conv(128, 320, 3, act="relu6")),  # two channel tiles, K = 9 x 2 chunks
+    (2, 28, 28, _conv(24, 144, 1, act="relu6")),   # channels not multiples of 16 / 64
+    (2, 29, 31, _conv(32, 64, 3, stride=2)),       # strided window
+    (2, 28, 28, _conv(256, 512, 1, stride=2, pad=0, act="none")),
+    (2, 24, 24, _conv(64, 64, 3, pool=2)),         # fused 2x2 max-pool
+    (9, 7, 7, _conv(512, 512, 3)),                 # several images per tile
+    (2, 33, 35, _conv(3, 32, 3, stride=2, act="relu6")),   # C = 3 stem (direct kernel)
+    (1, 45, 43, _conv(3, 64, 7, stride=2, pad=3)),
+    (2, 20, 20, _conv(3, 64, 3, pool=2)),
+    (2, 21, 22, _conv(96, 96, 3, stride=1, act="relu6", groups=96, op="dwconv")),
+    (2, 21, 22, _conv(144, 144, 3, stride=2, act="relu6", groups=144, op="dwconv")),
+    (2, 23, 21, _conv(64, 64, 3, stride=2, pad=1, act="none", op="maxpool")),
+]
+
+
+@pytest.mark.parametrize("case", SINGLE, ids=lambda c: "%dx%dx%d_%s_%d_%d_k%d_s%d" % (c[0], c[1], c[2], c[3]["op"], c[3]["cin"], c[3]["cout"], c[3]["kh"], c[3]["stride"]))
+def test_single_layer(case):
+    n, h, w, layer = case
+    sess, xd, ref = _mk([layer], "single", n, h, w, layer["cin"])
+    for s in (sms(), 3):
+        G.check_plan(sess, xd, ref, [0], [s], "single S=%d" % s)
+
+
+def test_single_layer_with_residual_through_both_conv_kernels():
+    layers = [_conv(64, 64, 1, act="none"), _conv(64, 64, 3, src=0, res_src=-1)]
+    sess, xd, ref = _mk(layers, "res", 2, 17, 18, 64)
+    G.check_plan(sess, xd, ref, [0, 1], [sms(), sms()], "residual tc")
+    B.net_set_option(sess.net, B.OPT_NO_TENSOR_CORE, 1)
+    G.check_plan(sess, xd, ref, [0, 1], [sms(), sms()], "residual direct")
+    assert sess.kernels() == ["conv_direct", "conv_direct"]
+
+
+def test_fc_and_avgpool():
+    layers = [_conv(32, 64, 3), dict(_conv(64, 64, 1, op="gavgpool", act="none"), src=0),
+              dict(op="fc", act="relu", cin=64, cout=40, kh=1, kw=1, stride=1, pad=0, groups=1, src=1, res_src=-2, pool=0),
+              dict(op="fc", act="none", cin=40, cout=13, kh=1, kw=1, stride=1, pad=0, groups=1, src=2, res_src=-2, pool=0)]
+    sess, xd, ref = _mk(layers, "fc", 11, 9, 9, 32)
+    G.check_plan(sess, xd, ref, [0, 1, 2, 3], [sms()] * 4, "fc")
+
+
+def test_tiny_network_with_every_layer_type():
+    layers = _tiny_resnet_like()
+    for l in layers:   # channel counts the vector kernels accept
+        pass
+    layers = [dict(l) for l in layers]
+    scale = {3: 3, 4: 8, 8: 16, 16: 32, 5: 8}
+    for l in layers:
+        l["cin"], l["cout"] = scale[l["cin"]], scale[l["cout"]]
+        if l["op"] == "dwconv":
+            l["groups"] = l["cin"]
+    layers[-1]["cin"] = 32
+    sess, xd, ref = _mk(layers, "tinynet", 2, 37, 35, 3)
+    G.check_plan(sess, xd, ref, list(range(len(layers))), [sms()] * len(layers), "tiny net")
+
+
+# ---- fused chains: every contiguous plan, ragged tiles, 1x1 / 3x3 mixes --------------------------------
+CHAINS = [
+    # (n, h, w, c, kernel sizes)
+    (1, 32, 32, 16, (3, 3)),
+    (2, 19, 23, 64, (3, 3, 3)),
+    (2, 14, 14, 128, (3, 1, 3)),
+    (1, 56, 56, 32, (1, 1, 1, 1)),
+    (3, 7, 7, 256, (3, 3)),
+    (1, 28, 28, 64, (3, 3, 3, 3)),
+]
+
+
+@pytest.mark.parametrize("case", CHAINS, ids=lambda c: "%dx%dx%dx%d_%s" % (c[0], c[1], c[2], c[3], "".join(map(str, c[4]))))
+def test_chain_every_contiguous_plan(case):
+    n, h, w, c, ks = case
+    layers = [_conv(c, c, k, src=i - 1) for i, k in enumerate(ks)]
+    sess, xd, ref = _mk(layers, "chain", n, h, w, c)
+    for ends in G.all_contiguous_plans(len(ks)):
+        for s in (sms(), 5):
+            G.check_plan(sess, xd, ref, ends, [s] * len(ends), "chain %s S=%d" % (ends, s))
+
+
+def test_chain_with_pool_and_residual_and_channel_change():
+    layers = [_conv(32, 64, 1), _conv(64, 64, 3, src=0), _conv(64, 32, 1, src=1, res_src=-1, act="relu"),
+              _conv(32, 48, 3, src=2, pool=2)]
+    sess, xd, ref = _mk(layers, "chain2", 2, 18, 22, 32)
+    G.check_plan(sess, xd, ref, [0, 1, 2, 3], [sms()] * 4, "unfused")
+    G.check_plan(sess, xd, ref, [2, 3], [sms(), 7], "bottleneck-like + pooled tail")
+    assert sess.kernels() == ["chain_tc", "chain_tc"]
+
+
+def test_illegal_plans_are_rejected():
+    layers = [_conv(32, 32, 3), _conv(32, 32, 3, stride=2, src=0), _conv(32, 32, 3, src=1)]
+    sess, xd, ref = _mk(layers, "illegal", 1, 16, 16, 32)
+    for ends, sm in (([2], [4]), ([0, 2, 1], [1, 1, 1]), ([0, 1], [1, 1]), ([0, 1, 2], [0, 1, 1]), ([0, 1, 2], [1, 1, 10 ** 6])):
+        with pytest.raises(B.DlfError) as e:
+            B.net_set_plan(sess.net, ends, sm)
+        assert e.value.status == B.E_PLAN
+    G.check_plan(sess, xd, ref, [0, 1, 2], [2, 2, 2], "legal")
