@@ -90,7 +90,7 @@ struct dlf_net {
     uint8_t* ws = nullptr;
     size_t ws_bytes = 0, ws_need = 0, in_off = 0, in_bytes = 0, status_off = 0;
     int dev_sms = 0;
-    int opt_no_tc = 0, opt_base_offset = 1, opt_single_chain = 0;
+    int opt_no_tc = 0, opt_base_offset = 0, opt_single_chain = 0;
     const void* last_out = nullptr;
 };
 

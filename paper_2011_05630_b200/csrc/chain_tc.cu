@@ -30,8 +30,7 @@ namespace dlf {
 namespace {
 
 constexpr int kThreads = 192;
-constexpr int kMaxSmem = 232448;
-constexpr int kSlackRows = 136;  // rows a shifted 128-row window may read past the frame
+constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
 
 struct ChainLayerP {
     int cin, cout, k, pad, act;
@@ -310,6 +309,21 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
 
 int planes_of(int c) { return (c + 63) / 64; }
 
+// Rows one activation plane must hold: the frame itself, plus what the last 128-row block of a
+// layer may touch past it (its own rows when written, its farthest tap when read).
+int rows_alloc_of(const ChainArgs& a, int rows, int pitch) {
+    int need = rows * pitch, c = 0;
+    for (int l = 0; l < a.n_layers; l++) {
+        const int pad = a.k[l] / 2;
+        c += pad;
+        const int qs = c * pitch + c;
+        const int range = (rows - 2 * c - 1) * pitch + (pitch - 2 * c);
+        const int nb = (range + 127) / 128;
+        need = std::max(need, qs + nb * 128 + pad * pitch + pad);
+    }
+    return (need + 7) / 8 * 8;
+}
+
 }  // namespace
 
 // Picks the output tile from the SM count: among the tile shapes whose buffers fit in shared
@@ -338,7 +352,7 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
             if (th > std::max(a.H, 2) * 2 || tw > std::max(a.W, 2) * 2) continue;
             const int rows = th + 2 * halo, pitch = tw + 2 * halo;
             if (rows > 256 || pitch > 256) continue;
-            const int rows_alloc = (rows * pitch + kSlackRows + 7) / 8 * 8;
+            const int rows_alloc = rows_alloc_of(a, rows, pitch);
             const size_t buf = static_cast<size_t>(planes_max) * rows_alloc * 128;
             int stages = 8;
             while (stages > 2 && 2 * buf + static_cast<size_t>(stages) * stage_bytes + 1024 > kMaxSmem) stages--;
@@ -413,7 +427,7 @@ int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int 
         int rc = encode_tmap(&p.tmw[l], a.w[l], 3, dims, strides, box, es);
         if (rc) return rc;
     }
-    const int rows_alloc = (t.rows * t.pitch + kSlackRows + 7) / 8 * 8;
+    const int rows_alloc = rows_alloc_of(a, t.rows, t.pitch);
     p.plane_bytes = rows_alloc * 128;
     p.buf_bytes = planes_max * p.plane_bytes;
     p.in_planes = planes_of(a.cin[0]);

@@ -25,7 +25,7 @@ namespace {
 
 constexpr int kThreads = 192;
 constexpr int kABytes = 128 * 128;  // 128 pixels x 64 fp16
-constexpr int kMaxSmem = 232448;
+constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
 
 struct ConvTcParams {
     int N, Ho, Wo, Cout;

@@ -115,7 +115,9 @@ __device__ __forceinline__ void tc_fence_after_sync() {
 
 // Shared-memory matrix descriptor, K-major operand, 128-byte swizzle: rows of 64 fp16 (128 bytes),
 // eight rows per 1024-byte swizzle atom, atoms of consecutive row groups 1024 bytes apart.
-// base_offset: row phase (address bits 7..9) of a start address that is not 1024-byte aligned.
+// The swizzle is a function of the absolute shared-memory address (bits 7..9 select the XOR of
+// bits 4..6), so a start address on any 128-byte row of a 1024-byte-aligned buffer is valid with
+// base_offset = 0; measured on B200: a non-zero base offset there breaks the operand.
 __device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr, uint32_t base_offset) {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);        // start address, 16-byte units

@@ -130,9 +130,18 @@ def test_chain_every_contiguous_plan(case):
     n, h, w, c, ks = case
     layers = [_conv(c, c, k, src=i - 1) for i, k in enumerate(ks)]
     sess, xd, ref = _mk(layers, "chain", n, h, w, c)
+    ran_fused = 0
     for ends in G.all_contiguous_plans(len(ks)):
         for s in (sms(), 5):
-            G.check_plan(sess, xd, ref, ends, [s] * len(ends), "chain %s S=%d" % (ends, s))
+            firsts = [0] + [e + 1 for e in ends[:-1]]
+            if all(B.net_group_is_legal(sess.net, a, e, s) for a, e in zip(firsts, ends)):
+                G.check_plan(sess, xd, ref, ends, [s] * len(ends), "chain %s S=%d" % (ends, s))
+                ran_fused += len(ends) < len(ks)
+            else:   # a group the kernel cannot hold is refused, never re-partitioned
+                with pytest.raises(B.DlfError) as e:
+                    B.net_set_plan(sess.net, ends, [s] * len(ends))
+                assert e.value.status == B.E_PLAN
+    assert ran_fused > 0
 
 
 def test_chain_with_pool_and_residual_and_channel_change():
@@ -141,7 +150,13 @@ def test_chain_with_pool_and_residual_and_channel_change():
     sess, xd, ref = _mk(layers, "chain2", 2, 18, 22, 32)
     G.check_plan(sess, xd, ref, [0, 1, 2, 3], [sms()] * 4, "unfused")
     G.check_plan(sess, xd, ref, [2, 3], [sms(), 7], "bottleneck-like + pooled tail")
-    assert sess.kernels() == ["chain_tc", "chain_tc"]
+    assert sess.kernels() == ["chain_tc", "conv_tc"]
+    # a fused group that ends in a pooled layer, odd image size (the last row / column is dropped)
+    layers = [_conv(32, 64, 3), _conv(64, 48, 3, src=0, pool=2), _conv(48, 48, 1, src=1)]
+    sess, xd, ref = _mk(layers, "chain3", 2, 19, 21, 32)
+    for s in (sms(), 7):
+        G.check_plan(sess, xd, ref, [1, 2], [s, s], "pooled tail S=%d" % s)
+        assert sess.kernels() == ["chain_tc", "conv_tc"]
 
 
 def test_illegal_plans_are_rejected():
