@@ -115,7 +115,7 @@ static int query_sms(int* out) {
 static bool chain_layer_ok(const Layer& l) {
     const dlf_layer_desc& d = l.d;
     return d.op == DLF_CONV && d.groups == 1 && d.stride == 1 && d.kh == d.kw && (d.kh == 1 || d.kh == 3) &&
-           d.pad == d.kh / 2 && d.cin % 8 == 0 && d.cout % 8 == 0 && d.cout <= 256;
+           d.pad == d.kh / 2 && chain_tc_layer_supported(d.cin, d.cout, d.kh);
 }
 
 static bool span_is_chain(const dlf_net* net, int first, int last) {

@@ -2,7 +2,8 @@
 // 1x1) with bias / activation after each, optional residual and 2x2 max-pool on the last one,
 // executed by ONE kernel whose intermediate feature maps never leave the SM (Sec. III-B of the
 // paper: a fused layer's output is produced on chip and reused at once; Sec. IV-B: a spatial
-// tile of a fused block recomputes its halo).
+// tile of a fused block recomputes its halo).  With one layer it is also the library's general
+// stride-1 convolution kernel: the input tile is read once instead of once per tap.
 //
 // Work item = (image, output tile th x tw of the last layer).  The tile's receptive-field frame
 // (th + 2 halo) x (tw + 2 halo), halo = sum of the paddings, is loaded ONCE by TMA (zero fill
@@ -12,15 +13,22 @@
 // rows, so every layer - the first included - feeds the tensor cores straight from the resident
 // tile through a shifted shared-memory descriptor: no im2col, no per-tap reload.  A layer's M
 // dimension is the linear range of frame positions it must produce (wrap-around columns are
-// computed and ignored); its accumulators (up to 512 TMEM columns) are drained by four epilogue
-// warps that add the bias, apply the activation, round to fp16, force positions outside the
-// image to zero (they are the next layer's padding) and write the next layer's operand tile back
-// to shared memory.  Weights stream through a TMA ring, once per layer per tile.
+// computed and ignored), cut into 128-row blocks; output channels are cut into chunks of at
+// most 256.  A pass = (layer, channel chunk, group of blocks) accumulates in one half of tensor
+// memory while the four epilogue warps drain the other half: bias, residual, activation, fp16
+// rounding, then either the next layer's operand tile in shared memory (positions outside the
+// image forced to zero: they are the next layer's padding) or, for the group's last layer,
+// global memory.  Weights stream through a TMA ring, once per pass; the next tile's input frame
+// is prefetched into a second buffer while the current tile computes.
+//
+// Warp roles: 0 weight producer, 1 UMMA issuer (owns the TMEM allocation), 2-5 epilogue,
+// 6 input producer.
 #include <cuda.h>
 #include <cuda_fp16.h>
 
 #include <algorithm>
 #include <cstring>
+#include <vector>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -29,16 +37,18 @@ namespace dlf {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;
 constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
+constexpr int kMaxBias = 4096;           // floats of bias staged in shared memory (all layers)
 
 struct ChainLayerP {
     int cin, cout, k, pad, act;
-    int n_pad;      // cout rounded up to 16 (UMMA N)
-    int slot;       // TMEM columns per 128-row block: n_pad rounded up to 32
-    int kchunks;    // ceil(cin / 64)
-    int ksteps_last;
-    int cum_pad;    // sum of paddings up to and including this layer
+    int kchunks, ksteps_last;  // 64-channel K chunks; 16-channel steps in the last one
+    int qs, range, nb;         // first frame row produced, rows produced, 128-row blocks
+    int n_pad;                 // cout rounded up to 16
+    int n_chunks, chunk_n;     // channel chunks of chunk_n (the last one may be smaller)
+    int slot, per_pass;        // TMEM columns per block, blocks per pass (half of TMEM)
+    int bias_off;
     const float* bias;
 };
 
@@ -51,9 +61,10 @@ struct ChainParams {
     int th, tw, halo, pitch, rows;  // frame geometry
     int tiles_h, tiles_w, n_tiles;
     int plane_bytes;                // rows_alloc * 128
-    int buf_bytes;                  // planes_max * plane_bytes
-    int in_planes;
-    int stages, stage_bytes;
+    int in_planes, in_bufs, in_buf_bytes;
+    int act_off, act_buf_bytes;
+    int ring_off, stages, stage_bytes;
+    int bias_off, bias_floats;
     int pool, base_offset_mode;
     int cout_last;
     const __half* res;
@@ -63,16 +74,20 @@ struct ChainParams {
 
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+__device__ __forceinline__ int chunk_cols(const ChainLayerP& L, int c) {
+    return min(L.chunk_n, L.n_pad - c * L.chunk_n);
+}
+
 __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t wfull_bar[8], wempty_bar[8], in_full_bar, in_empty_bar, acc_full_bar, epi_done_bar;
+    __shared__ uint64_t wfull_bar[8], wempty_bar[8], in_full_bar[2], in_empty_bar[2], acc_full_bar[2], acc_empty_bar[2],
+        act_ready_bar;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
-    // layout: [buf0][buf1][weight ring]
-    const uint32_t ring_off = 2u * p.buf_bytes;
+    float* bias_s = reinterpret_cast<float*>(sbase + p.bias_off);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &abort_s;
 
@@ -82,10 +97,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             mbar_init(&wfull_bar[i], 1);
             mbar_init(&wempty_bar[i], 1);
         }
-        mbar_init(&in_full_bar, 1);
-        mbar_init(&in_empty_bar, 1);
-        mbar_init(&acc_full_bar, 1);
-        mbar_init(&epi_done_bar, 4);
+        for (int i = 0; i < 2; i++) {
+            mbar_init(&in_full_bar[i], 1);
+            mbar_init(&in_empty_bar[i], 1);
+            mbar_init(&acc_full_bar[i], 1);
+            mbar_init(&acc_empty_bar[i], 4);
+        }
+        mbar_init(&act_ready_bar, 4);
         fence_barrier_init();
         tma_prefetch_desc(&p.tmx);
     }
@@ -93,98 +111,109 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         tmem_alloc(&tmem_base_s, 512);
         tmem_relinquish();
     }
+    for (int l = 0; l < p.n_layers; l++) {
+        const ChainLayerP& L = p.L[l];
+        for (int i = threadIdx.x; i < L.n_pad; i += kThreads) bias_s[L.bias_off + i] = i < L.cout ? __ldg(L.bias + i) : 0.0f;
+    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = tmem_base_s;
     const int frame_rows = p.rows * p.pitch;
 
-    if (warp == 0) {
-        // ---- producer ----------------------------------------------------------------------------------
+    if (warp == 6) {
+        // ---- input producer: one frame per tile, prefetched into the free input buffer ---------
         if (lane == 0) {
-            uint32_t wit = 0, tile_i = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x, tile_i++) {
+            uint32_t tile_i = 0;
+            for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x, tile_i++) {
                 const int txi = t % p.tiles_w, tyi = (t / p.tiles_w) % p.tiles_h, n = t / (p.tiles_w * p.tiles_h);
-                ok = mbar_wait(&in_empty_bar, (tile_i & 1u) ^ 1u, abort_flag, p.status, 0x100 | (blockIdx.x << 12));
-                if (!ok) break;
-                mbar_expect_tx(&in_full_bar, static_cast<uint32_t>(p.in_planes) * frame_rows * 128u);
+                const uint32_t ib = tile_i % p.in_bufs, ph = (tile_i / p.in_bufs) & 1u;
+                if (!mbar_wait(&in_empty_bar[ib], ph ^ 1u, abort_flag, p.status, 0x100 | (blockIdx.x << 12))) break;
+                mbar_expect_tx(&in_full_bar[ib], static_cast<uint32_t>(p.in_planes) * frame_rows * 128u);
                 for (int pl = 0; pl < p.in_planes; pl++)
-                    tma_load_4d(sbase + static_cast<size_t>(pl) * p.plane_bytes, &p.tmx, &in_full_bar, pl * 64,
-                                txi * p.tw - p.halo, tyi * p.th - p.halo, n);
+                    tma_load_4d(sbase + static_cast<size_t>(ib) * p.in_buf_bytes + static_cast<size_t>(pl) * p.plane_bytes, &p.tmx,
+                                &in_full_bar[ib], pl * 64, txi * p.tw - p.halo, tyi * p.th - p.halo, n);
+            }
+        }
+    } else if (warp == 0) {
+        // ---- weight producer: one [chunk_n][64] slab per (tap, K chunk) of every pass ---------------
+        if (lane == 0) {
+            uint32_t wit = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
                 for (int l = 0; l < p.n_layers && ok; l++) {
                     const ChainLayerP& L = p.L[l];
-                    const int c = L.cum_pad;
-                    const int range = (p.rows - 2 * c - 1) * p.pitch + (p.pitch - 2 * c);
-                    const int nb = (range + 127) / 128, per_pass = 512 / L.slot;
-                    const int passes = (nb + per_pass - 1) / per_pass;
-                    const uint32_t bytes = static_cast<uint32_t>(L.n_pad) * 128u;
-                    for (int ps = 0; ps < passes && ok; ps++)
-                        for (int tap = 0; tap < L.k * L.k && ok; tap++)
-                            for (int kc = 0; kc < L.kchunks; kc++, wit++) {
-                                const int st = wit % p.stages;
-                                ok = mbar_wait(&wempty_bar[st], ((wit / p.stages) & 1u) ^ 1u, abort_flag, p.status,
-                                               0x200 | (blockIdx.x << 12));
-                                if (!ok) break;
-                                mbar_expect_tx(&wfull_bar[st], bytes);
-                                tma_load_3d(sbase + ring_off + static_cast<size_t>(st) * p.stage_bytes, &p.tmw[l],
-                                            &wfull_bar[st], kc * 64, tap, 0);
-                            }
+                    const int passes = (L.nb + L.per_pass - 1) / L.per_pass;
+                    for (int c = 0; c < L.n_chunks && ok; c++) {
+                        const uint32_t bytes = static_cast<uint32_t>(L.chunk_n) * 128u;  // the whole box, rows past cout zero-filled
+                        for (int ps = 0; ps < passes && ok; ps++)
+                            for (int tap = 0; tap < L.k * L.k && ok; tap++)
+                                for (int kc = 0; kc < L.kchunks; kc++, wit++) {
+                                    const int st = wit % p.stages;
+                                    ok = mbar_wait(&wempty_bar[st], ((wit / p.stages) & 1u) ^ 1u, abort_flag, p.status,
+                                                   0x200 | (blockIdx.x << 12));
+                                    if (!ok) break;
+                                    mbar_expect_tx(&wfull_bar[st], bytes);
+                                    tma_load_3d(sbase + p.ring_off + static_cast<size_t>(st) * p.stage_bytes, &p.tmw[l],
+                                                &wfull_bar[st], kc * 64, tap, c * L.chunk_n);
+                                }
+                    }
                 }
             }
         }
     } else if (warp == 1) {
-        // ---- MMA issuer -----------------------------------------------------------------------------------
+        // ---- UMMA issuer ------------------------------------------------------------------------------------
         if (lane == 0) {
-            uint32_t wit = 0, tile_i = 0, pass_i = 0;
+            uint32_t wit = 0, tile_i = 0, pass_i = 0, act_i = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x, tile_i++) {
-                ok = mbar_wait(&in_full_bar, tile_i & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
+                const uint32_t ib = tile_i % p.in_bufs;
+                ok = mbar_wait(&in_full_bar[ib], (tile_i / p.in_bufs) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                 if (!ok) break;
                 for (int l = 0; l < p.n_layers && ok; l++) {
                     const ChainLayerP& L = p.L[l];
-                    const int c = L.cum_pad;
-                    const int qs = c * p.pitch + c;
-                    const int range = (p.rows - 2 * c - 1) * p.pitch + (p.pitch - 2 * c);
-                    const int nb = (range + 127) / 128, per_pass = 512 / L.slot;
-                    const uint32_t idesc = umma_idesc_f16(L.n_pad);
-                    const uint32_t abuf = base + (l & 1) * p.buf_bytes;
-                    for (int b0 = 0; b0 < nb && ok; b0 += per_pass, pass_i++) {
-                        const int nblk = min(per_pass, nb - b0);
-                        if (pass_i > 0) {
-                            // previous pass drained: TMEM is free and its shared-memory output is visible
-                            ok = mbar_wait(&epi_done_bar, (pass_i - 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
+                    if (l > 0) {  // the epilogue has written all of the previous layer's tile
+                        ok = mbar_wait(&act_ready_bar, act_i & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
+                        if (!ok) break;
+                        act_i++;
+                    }
+                    const uint32_t abuf = l == 0 ? base + ib * p.in_buf_bytes : base + p.act_off + ((l - 1) & 1) * p.act_buf_bytes;
+                    for (int c = 0; c < L.n_chunks && ok; c++) {
+                        const uint32_t idesc = umma_idesc_f16(chunk_cols(L, c));
+                        for (int b0 = 0; b0 < L.nb && ok; b0 += L.per_pass, pass_i++) {
+                            const int nblk = min(L.per_pass, L.nb - b0);
+                            const uint32_t half = pass_i & 1u;
+                            ok = mbar_wait(&acc_empty_bar[half], ((pass_i >> 1) & 1u) ^ 1u, abort_flag, p.status,
+                                           0x500 | (blockIdx.x << 12));
                             if (!ok) break;
-                        }
-                        tc_fence_after_sync();
-                        for (int tap = 0; tap < L.k * L.k && ok; tap++) {
-                            const int r = tap / L.k, s = tap % L.k;
-                            const int shift = (r - L.pad) * p.pitch + (s - L.pad);
-                            for (int kc = 0; kc < L.kchunks; kc++, wit++) {
-                                const int st = wit % p.stages;
-                                ok = mbar_wait(&wfull_bar[st], (wit / p.stages) & 1u, abort_flag, p.status,
-                                               0x500 | (blockIdx.x << 12));
-                                if (!ok) break;
-                                tc_fence_after_sync();
-                                const uint32_t wsm = base + ring_off + st * p.stage_bytes;
-                                const int ksteps = (kc == L.kchunks - 1) ? L.ksteps_last : 4;
-                                for (int b = 0; b < nblk; b++) {
-                                    const uint32_t arow = abuf + kc * p.plane_bytes + (qs + (b0 + b) * 128 + shift) * 128;
-                                    const uint32_t bo = p.base_offset_mode ? ((arow >> 7) & 7u) : 0u;
-                                    const uint32_t d_tmem = tmem_base + b * L.slot;
-                                    for (int ks = 0; ks < ksteps; ks++)
-                                        umma_f16(d_tmem, umma_desc_sw128(arow + ks * 32, bo),
-                                                 umma_desc_sw128(wsm + ks * 32, 0), idesc, (tap | kc | ks) != 0);
+                            tc_fence_after_sync();
+                            for (int tap = 0; tap < L.k * L.k && ok; tap++) {
+                                const int r = tap / L.k, s = tap % L.k;
+                                const int shift = (r - L.pad) * p.pitch + (s - L.pad);
+                                for (int kc = 0; kc < L.kchunks; kc++, wit++) {
+                                    const int st = wit % p.stages;
+                                    ok = mbar_wait(&wfull_bar[st], (wit / p.stages) & 1u, abort_flag, p.status,
+                                                   0x600 | (blockIdx.x << 12));
+                                    if (!ok) break;
+                                    tc_fence_after_sync();
+                                    const uint32_t wsm = base + p.ring_off + st * p.stage_bytes;
+                                    const int ksteps = (kc == L.kchunks - 1) ? L.ksteps_last : 4;
+                                    for (int b = 0; b < nblk; b++) {
+                                        const uint32_t arow = abuf + kc * p.plane_bytes + (L.qs + (b0 + b) * 128 + shift) * 128;
+                                        const uint32_t bo = p.base_offset_mode ? ((arow >> 7) & 7u) : 0u;
+                                        const uint32_t d_tmem = tmem_base + half * 256u + b * L.slot;
+                                        for (int ks = 0; ks < ksteps; ks++)
+                                            umma_f16(d_tmem, umma_desc_sw128(arow + ks * 32, bo),
+                                                     umma_desc_sw128(wsm + ks * 32, 0), idesc, (tap | kc | ks) != 0);
+                                    }
+                                    umma_commit(&wempty_bar[st]);
                                 }
-                                umma_commit(&wempty_bar[st]);
                             }
-                        }
-                        if (ok) {
-                            umma_commit(&acc_full_bar);
-                            // an odd-length chain reads the input buffer last in its final layer
-                            if (l == p.n_layers - 1 && b0 + per_pass >= nb && (p.n_layers & 1)) umma_commit(&in_empty_bar);
+                            if (ok) umma_commit(&acc_full_bar[half]);
                         }
                     }
+                    // the input frame is read by the first layer only
+                    if (ok && l == 0) umma_commit(&in_empty_bar[ib]);
                 }
             }
         }
@@ -201,73 +230,101 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             for (int l = 0; l < p.n_layers && ok; l++) {
                 const ChainLayerP& L = p.L[l];
                 const bool last = (l == p.n_layers - 1);
-                const int c = L.cum_pad;
-                const int qs = c * p.pitch + c;
-                const int range = (p.rows - 2 * c - 1) * p.pitch + (p.pitch - 2 * c);
-                const int nb = (range + 127) / 128, per_pass = 512 / L.slot;
-                uint8_t* obuf = sbase + ((l + 1) & 1) * p.buf_bytes;
-                for (int b0 = 0; b0 < nb && ok; b0 += per_pass, pass_i++) {
-                    const int nblk = min(per_pass, nb - b0);
-                    ok = mbar_wait(&acc_full_bar, pass_i & 1u, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    for (int b = 0; b < nblk; b++) {
-                        const int q = qs + (b0 + b) * 128 + row;
-                        const int fy = q / p.pitch, fx = q - fy * p.pitch;
-                        const int gy = gy0 + fy, gx = gx0 + fx;
-                        const bool in_range = q < qs + range;
-                        const bool in_img = gy >= 0 && gy < p.H && gx >= 0 && gx < p.W;
-                        const long long gpix = (static_cast<long long>(n) * p.H + gy) * p.W + gx;
-                        const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + b * L.slot;
-                        for (int cc = 0; cc < L.n_pad; cc += 16) {
-                            float v[16];
-                            __syncwarp();  // the aligned TMEM load needs the whole warp converged
-                            tmem_ld16(taddr + cc, v);
-                            if (!in_range) continue;
-                            uint32_t packed[8];
+                const bool to_global = last && !p.pool;
+                uint8_t* obuf = sbase + p.act_off + (l & 1) * p.act_buf_bytes;
+                const float* bl = bias_s + L.bias_off;
+                for (int c = 0; c < L.n_chunks && ok; c++) {
+                    const int ncols = chunk_cols(L, c), ch0 = c * L.chunk_n;
+                    for (int b0 = 0; b0 < L.nb && ok; b0 += L.per_pass, pass_i++) {
+                        const int nblk = min(L.per_pass, L.nb - b0);
+                        const uint32_t half = pass_i & 1u;
+                        ok = mbar_wait(&acc_full_bar[half], (pass_i >> 1) & 1u, abort_flag, p.status, 0x700 | (blockIdx.x << 12));
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        for (int b = 0; b < nblk; b++) {
+                            const int q = L.qs + (b0 + b) * 128 + row;
+                            const int fy = q / p.pitch, fx = q - fy * p.pitch;
+                            const int gy = gy0 + fy, gx = gx0 + fx;
+                            const bool in_range = q < L.qs + L.range;
+                            const bool in_img = gy >= 0 && gy < p.H && gx >= 0 && gx < p.W;
+                            const bool in_tile = fy >= p.halo && fy < p.halo + p.th && fx >= p.halo && fx < p.halo + p.tw;
+                            const long long gpix = (static_cast<long long>(n) * p.H + gy) * p.W + gx;
+                            const bool live = in_range && (to_global ? (in_img && in_tile) : true);
+                            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + half * 256u + b * L.slot;
+                            for (int cc = 0; cc < ncols; cc += 32) {
+                                float v[32];
+                                __syncwarp();  // the aligned TMEM loads need the whole warp converged
+                                const int nc = min(32, ncols - cc);
+                                if (nc == 32) tmem_ld32(taddr + cc, v);
+                                else tmem_ld16(taddr + cc, v);
+                                if (!live) continue;
+                                for (int h = 0; h < nc; h += 16) {
+                                    const int co = ch0 + cc + h;  // first of 16 channels
+                                    uint32_t packed[8];
+                                    if (in_img) {
+                                        float a[16];
 #pragma unroll
-                            for (int e = 0; e < 8; e++) {
-                                const int co = cc + 2 * e;
-                                float a0 = 0.0f, a1 = 0.0f;
-                                if (in_img && co < L.cout) {  // cout is a multiple of 8: pairs never straddle
-                                    a0 = v[2 * e] + __ldg(L.bias + co);
-                                    a1 = v[2 * e + 1] + __ldg(L.bias + co + 1);
-                                    if (last && p.res != nullptr) {
-                                        const __half2 rh = __ldg(reinterpret_cast<const __half2*>(p.res + gpix * L.cout + co));
-                                        const float2 rf = __half22float2(rh);
-                                        a0 += rf.x;
-                                        a1 += rf.y;
+                                        for (int e = 0; e < 16; e += 4) {
+                                            const float4 bb = *reinterpret_cast<const float4*>(bl + co + e);
+                                            a[e] = v[h + e] + bb.x; a[e + 1] = v[h + e + 1] + bb.y;
+                                            a[e + 2] = v[h + e + 2] + bb.z; a[e + 3] = v[h + e + 3] + bb.w;
+                                        }
+                                        if (last && p.res != nullptr) {
+#pragma unroll
+                                            for (int g = 0; g < 2; g++) {
+                                                if (co + g * 8 < L.cout) {
+                                                    const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.res + gpix * L.cout + co + g * 8));
+                                                    const __half2* rh = reinterpret_cast<const __half2*>(&rv);
+#pragma unroll
+                                                    for (int e = 0; e < 4; e++) {
+                                                        const float2 rf = __half22float2(rh[e]);
+                                                        a[g * 8 + 2 * e] += rf.x;
+                                                        a[g * 8 + 2 * e + 1] += rf.y;
+                                                    }
+                                                }
+                                            }
+                                        }
+#pragma unroll
+                                        for (int e = 0; e < 8; e++)
+                                            packed[e] = pack_half2(apply_act(a[2 * e], L.act), apply_act(a[2 * e + 1], L.act));
+                                        // channels past cout (padding up to 16) carry zero weights and zero bias:
+                                        // act(0) = 0, so the next layer's K padding stays zero
+                                    } else {
+#pragma unroll
+                                        for (int e = 0; e < 8; e++) packed[e] = 0u;
                                     }
-                                    a0 = apply_act(a0, L.act);
-                                    a1 = apply_act(a1, L.act);
-                                }
-                                packed[e] = pack_half2(a0, a1);
-                            }
 #pragma unroll
-                            for (int h8 = 0; h8 < 2; h8++) {
-                                const int g8 = (cc >> 3) + h8;  // 8-channel group index
-                                uint8_t* dst = obuf + static_cast<size_t>(g8 >> 3) * p.plane_bytes + static_cast<size_t>(q) * 128 +
-                                               (((g8 & 7) ^ (q & 7)) << 4);
-                                *reinterpret_cast<uint4*>(dst) =
-                                    make_uint4(packed[h8 * 4], packed[h8 * 4 + 1], packed[h8 * 4 + 2], packed[h8 * 4 + 3]);
+                                    for (int g = 0; g < 2; g++) {
+                                        const uint4 val = make_uint4(packed[g * 4], packed[g * 4 + 1], packed[g * 4 + 2], packed[g * 4 + 3]);
+                                        if (to_global) {
+                                            if (co + g * 8 < L.cout)
+                                                *reinterpret_cast<uint4*>(p.out + gpix * L.cout + co + g * 8) = val;
+                                        } else {
+                                            const int g8 = (co >> 3) + g;  // 8-channel group index
+                                            uint8_t* dst = obuf + static_cast<size_t>(g8 >> 3) * p.plane_bytes +
+                                                           static_cast<size_t>(q) * 128 + (((g8 & 7) ^ (q & 7)) << 4);
+                                            *reinterpret_cast<uint4*>(dst) = val;
+                                        }
+                                    }
+                                }
                             }
                         }
+                        if (!to_global) fence_proxy_async_smem();  // UMMA reads these rows through the async proxy
+                        tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&acc_empty_bar[half]);
                     }
-                    fence_proxy_async_smem();  // the next layer's UMMAs read these rows through the async proxy
-                    tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&epi_done_bar);
                 }
+                if (ok && !last && lane == 0) mbar_arrive(&act_ready_bar);
             }
             if (!ok) break;
-            // ---- copy the tile out (coalesced 16-byte stores), pooling 2x2 if asked ----------------
-            epi_bar_sync();
-            {
-                const uint8_t* obuf = sbase + (p.n_layers & 1) * p.buf_bytes;
+            if (p.pool) {
+                // ---- pooled copy-out from the staging buffer (coalesced 16-byte stores) -----------------
+                epi_bar_sync();
+                const uint8_t* obuf = sbase + p.act_off + ((p.n_layers - 1) & 1) * p.act_buf_bytes;
                 const int c8n = p.cout_last / 8;
-                const int win = p.pool ? 2 : 1;
-                const int oth = p.th / win, otw = p.tw / win;
-                const int Ho = p.H / win, Wo = p.W / win;
+                const int oth = p.th / 2, otw = p.tw / 2;
+                const int Ho = p.H / 2, Wo = p.W / 2;
                 const int total = oth * otw * c8n;
                 for (int i = et; i < total; i += 128) {
                     const int g8 = i % c8n;
@@ -275,39 +332,55 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                     const int gy = tyi * oth + oy, gx = txi * otw + ox;
                     if (gy >= Ho || gx >= Wo) continue;
                     uint4 best = make_uint4(0, 0, 0, 0);
-                    for (int wy = 0; wy < win; wy++)
-                        for (int wx = 0; wx < win; wx++) {
-                            const int q = (p.halo + oy * win + wy) * p.pitch + p.halo + ox * win + wx;
-                            const uint4 vv = *reinterpret_cast<const uint4*>(obuf + static_cast<size_t>(g8 >> 3) * p.plane_bytes +
-                                                                             static_cast<size_t>(q) * 128 + (((g8 & 7) ^ (q & 7)) << 4));
-                            if (wy == 0 && wx == 0) {
-                                best = vv;
-                            } else {
-                                __half2* bh = reinterpret_cast<__half2*>(&best);
-                                const __half2* vh = reinterpret_cast<const __half2*>(&vv);
 #pragma unroll
-                                for (int e = 0; e < 4; e++) bh[e] = __hmax2(bh[e], vh[e]);
-                            }
+                    for (int wq = 0; wq < 4; wq++) {
+                        const int q = (p.halo + oy * 2 + (wq >> 1)) * p.pitch + p.halo + ox * 2 + (wq & 1);
+                        const uint4 vv = *reinterpret_cast<const uint4*>(obuf + static_cast<size_t>(g8 >> 3) * p.plane_bytes +
+                                                                         static_cast<size_t>(q) * 128 + (((g8 & 7) ^ (q & 7)) << 4));
+                        if (wq == 0) {
+                            best = vv;
+                        } else {
+                            __half2* bh = reinterpret_cast<__half2*>(&best);
+                            const __half2* vh = reinterpret_cast<const __half2*>(&vv);
+#pragma unroll
+                            for (int e = 0; e < 4; e++) bh[e] = __hmax2(bh[e], vh[e]);
                         }
+                    }
                     *reinterpret_cast<uint4*>(p.out + ((static_cast<long long>(n) * Ho + gy) * Wo + gx) * p.cout_last + g8 * 8) = best;
                 }
+                epi_bar_sync();
             }
-            epi_bar_sync();
-            // an even-length chain overwrites the input buffer in its last epilogue
-            if (!(p.n_layers & 1) && et == 0) mbar_arrive(&in_empty_bar);
         }
     }
 
     tc_fence_before_sync();
     __syncthreads();
     if (warp == 1) {
-        if (abort_s) __nanosleep(20000);
+        if (abort_s) __nanosleep(20000);  // let copies in flight land before the CTA retires
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, 512);
     }
 }
 
 int planes_of(int c) { return (c + 63) / 64; }
+int pad16(int c) { return (c + 15) / 16 * 16; }
+
+struct LayerGeom {
+    int qs, range, nb, n_pad, n_chunks, chunk_n, slot, per_pass;
+};
+
+LayerGeom layer_geom(int cout, int cum_pad, int rows, int pitch) {
+    LayerGeom g;
+    g.qs = cum_pad * pitch + cum_pad;
+    g.range = (rows - 2 * cum_pad - 1) * pitch + (pitch - 2 * cum_pad);
+    g.nb = (g.range + 127) / 128;
+    g.n_pad = pad16(cout);
+    g.n_chunks = (g.n_pad + 255) / 256;
+    g.chunk_n = g.n_chunks == 1 ? g.n_pad : 256;
+    g.slot = (std::min(g.chunk_n, g.n_pad) + 31) / 32 * 32;
+    g.per_pass = 256 / g.slot;
+    return g;
+}
 
 // Rows one activation plane must hold: the frame itself, plus what the last 128-row block of a
 // layer may touch past it (its own rows when written, its farthest tap when read).
@@ -316,76 +389,104 @@ int rows_alloc_of(const ChainArgs& a, int rows, int pitch) {
     for (int l = 0; l < a.n_layers; l++) {
         const int pad = a.k[l] / 2;
         c += pad;
-        const int qs = c * pitch + c;
-        const int range = (rows - 2 * c - 1) * pitch + (pitch - 2 * c);
-        const int nb = (range + 127) / 128;
-        need = std::max(need, qs + nb * 128 + pad * pitch + pad);
+        const LayerGeom g = layer_geom(a.cout[l], c, rows, pitch);
+        need = std::max(need, g.qs + g.nb * 128 + pad * pitch + pad);
     }
     return (need + 7) / 8 * 8;
 }
 
+std::vector<int> tile_candidates(int extent, bool even) {
+    std::vector<int> v;
+    for (int parts = 1; parts <= 16; parts++) {
+        int t = (extent + parts - 1) / parts;
+        if (even) t = (t + 1) / 2 * 2;
+        if (t >= 1) v.push_back(t);
+    }
+    for (int t : {2, 4, 8, 16, 32, 64}) v.push_back(t);
+    std::sort(v.begin(), v.end());
+    v.erase(std::unique(v.begin(), v.end()), v.end());
+    return v;
+}
+
 }  // namespace
 
-// Picks the output tile from the SM count: among the tile shapes whose buffers fit in shared
-// memory, the one with the least estimated time = waves x (tensor-core work of one tile,
-// counted in 128-row blocks, plus a fixed per-tile cost).
+bool chain_tc_layer_supported(int cin, int cout, int k) {
+    return (k == 1 || k == 3) && cin % 8 == 0 && cout % 8 == 0 && cin >= 8 && cout >= 8 && cout <= 2048 && cin <= 1024;
+}
+
+// Picks the output tile from the SM count (Sec. IV-B: more cores -> smaller tiles -> more
+// recomputed halo).  Among the tile shapes whose buffers fit in shared memory, takes the least
+// estimated time = waves x per-tile time, the per-tile time being modelled in SM clocks from the
+// UMMA issue rate (operand reads from shared memory vs. math), the epilogue and the input load.
 ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
     ChainTiling best{};
     best.ok = false;
     (void)device_sms;
-    if (a.n_layers < 1 || a.n_layers > kMaxChain) return best;
-    int halo = 0, planes_max = 0, nmax = 0;
+    if (a.n_layers < 1 || a.n_layers > kMaxChain || sm_count < 1) return best;
+    int halo = 0, bias_floats = 0, stage_n = 0;
     for (int l = 0; l < a.n_layers; l++) {
-        if (a.k[l] != 1 && a.k[l] != 3) return best;
-        if (a.cin[l] % 8 || a.cout[l] % 8 || a.cout[l] > 256) return best;
+        if (!chain_tc_layer_supported(a.cin[l], a.cout[l], a.k[l])) return best;
         if (l > 0 && a.cin[l] != a.cout[l - 1]) return best;
         halo += a.k[l] / 2;
-        planes_max = std::max(planes_max, std::max(planes_of(a.cin[l]), planes_of((a.cout[l] + 15) / 16 * 16)));
-        nmax = std::max(nmax, (a.cout[l] + 15) / 16 * 16);
+        bias_floats += pad16(a.cout[l]);
+        stage_n = std::max(stage_n, std::min(pad16(a.cout[l]), 256));
     }
-    const int stage_bytes = nmax * 128;
-    static const int cand[] = {2, 4, 6, 8, 12, 16, 24, 32, 48, 64};
-    double best_cost = -1.0;
-    for (int th : cand)
-        for (int tw : cand) {
-            if (a.pool && ((th | tw) & 1)) continue;
-            if (th > std::max(a.H, 2) * 2 || tw > std::max(a.W, 2) * 2) continue;
+    if (bias_floats > kMaxBias) return best;
+    const int L = a.n_layers;
+    const int stage_bytes = stage_n * 128;
+    const int in_planes = planes_of(a.cin[0]);
+    int act_bufs = (L == 1) ? (a.pool ? 1 : 0) : ((L == 2 && !a.pool) ? 1 : 2);
+    int act_planes = 0;
+    for (int l = 0; l < L; l++)
+        if (l < L - 1 || a.pool) act_planes = std::max(act_planes, planes_of(pad16(a.cout[l])));
+    const std::vector<int> cand_h = tile_candidates(a.H, a.pool != 0), cand_w = tile_candidates(a.W, a.pool != 0);
+    for (int th : cand_h)
+        for (int tw : cand_w) {
             const int rows = th + 2 * halo, pitch = tw + 2 * halo;
             if (rows > 256 || pitch > 256) continue;
             const int rows_alloc = rows_alloc_of(a, rows, pitch);
-            const size_t buf = static_cast<size_t>(planes_max) * rows_alloc * 128;
-            int stages = 8;
-            while (stages > 2 && 2 * buf + static_cast<size_t>(stages) * stage_bytes + 1024 > kMaxSmem) stages--;
-            if (2 * buf + static_cast<size_t>(stages) * stage_bytes + 1024 > kMaxSmem) continue;
+            const size_t plane = static_cast<size_t>(rows_alloc) * 128;
+            const size_t fixed = static_cast<size_t>(act_bufs) * act_planes * plane + static_cast<size_t>(bias_floats) * 4 + 1024;
             const int tiles_h = (a.H + th - 1) / th, tiles_w = (a.W + tw - 1) / tw;
             const long long n_tiles = static_cast<long long>(a.N) * tiles_h * tiles_w;
             if (n_tiles > 0x7fffffffLL) continue;
             const long long waves = (n_tiles + sm_count - 1) / sm_count;
-            double work = 0.0, useful = 0.0, computed = 0.0;
-            int c = 0;
-            for (int l = 0; l < a.n_layers; l++) {
-                c += a.k[l] / 2;
-                const int range = (rows - 2 * c - 1) * pitch + (pitch - 2 * c);
-                const int nb = (range + 127) / 128;
-                const double kk = static_cast<double>(a.k[l]) * a.k[l] * ((a.cin[l] + 15) / 16 * 16);
-                const int npad = (a.cout[l] + 15) / 16 * 16;
-                const int slot = (npad + 31) / 32 * 32;
-                const int passes = (nb + 512 / slot - 1) / (512 / slot);
-                work += nb * 128.0 * kk * npad + passes * 2.0e5;
-                computed += nb * 128.0 * kk * npad;
-                useful += static_cast<double>(std::min(th, a.H)) * std::min(tw, a.W) * a.k[l] * a.k[l] * a.cin[l] * a.cout[l];
-            }
-            work += static_cast<double>(rows) * pitch * planes_max * 64 * 40.0 + 4.0e5;  // input load + fixed cost
-            const double cost = static_cast<double>(waves) * work;
-            if (best_cost < 0 || cost < best_cost) {
-                best_cost = cost;
-                best.th = th; best.tw = tw; best.halo = halo; best.pitch = pitch; best.rows = rows;
-                best.tiles_h = tiles_h; best.tiles_w = tiles_w; best.n_tiles = static_cast<int>(n_tiles);
-                best.stages = stages;
-                best.smem_bytes = 2 * buf + static_cast<size_t>(stages) * stage_bytes + 1024;
-                best.tmem_cols = 512;
-                best.redundancy = computed / useful;
-                best.ok = true;
+            for (int in_bufs = 2; in_bufs >= 1; in_bufs--) {
+                int stages = 6;
+                auto total = [&](int st) { return fixed + static_cast<size_t>(in_bufs) * in_planes * plane + static_cast<size_t>(st) * stage_bytes; };
+                while (stages > 2 && total(stages) > static_cast<size_t>(kMaxSmem)) stages--;
+                if (total(stages) > static_cast<size_t>(kMaxSmem)) continue;
+                double clk = 1500.0, useful = 0.0, computed = 0.0;
+                int c = 0;
+                for (int l = 0; l < L; l++) {
+                    c += a.k[l] / 2;
+                    const LayerGeom g = layer_geom(a.cout[l], c, rows, pitch);
+                    const int ksteps = a.k[l] * a.k[l] * ((a.cin[l] + 15) / 16);
+                    double mma = 0.0;
+                    for (int ch = 0; ch < g.n_chunks; ch++) {
+                        const int n = std::min(g.chunk_n, g.n_pad - ch * g.chunk_n);
+                        mma += static_cast<double>(g.nb) * ksteps * std::max(32.0 + n / 4.0, n / 2.0);
+                    }
+                    const double epi = static_cast<double>(g.nb) * (g.n_pad / 32.0) * 220.0;
+                    const int passes = g.n_chunks * ((g.nb + g.per_pass - 1) / g.per_pass);
+                    clk += (passes > 1 ? std::max(mma, epi) + std::min(mma, epi) / passes : mma + epi) + 600.0;
+                    computed += static_cast<double>(g.nb) * 128.0 * a.k[l] * a.k[l] * a.cin[l] * a.cout[l];
+                    useful += static_cast<double>(std::min(th, a.H)) * std::min(tw, a.W) * a.k[l] * a.k[l] * a.cin[l] * a.cout[l];
+                }
+                const double load = static_cast<double>(rows) * pitch * in_planes * 128.0 / 48.0;
+                clk = (in_bufs == 2) ? std::max(clk, load) : clk + load + 1500.0;
+                const double cost = static_cast<double>(waves) * clk;
+                if (!best.ok || cost < best.cost) {
+                    best.th = th; best.tw = tw; best.halo = halo; best.pitch = pitch; best.rows = rows;
+                    best.rows_alloc = rows_alloc;
+                    best.tiles_h = tiles_h; best.tiles_w = tiles_w; best.n_tiles = static_cast<int>(n_tiles);
+                    best.in_bufs = in_bufs; best.act_bufs = act_bufs; best.act_planes = act_planes;
+                    best.stages = stages; best.stage_bytes = stage_bytes;
+                    best.smem_bytes = total(stages);
+                    best.redundancy = computed / useful;
+                    best.cost = cost;
+                    best.ok = true;
+                }
             }
         }
     return best;
@@ -406,33 +507,38 @@ int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int 
     p.N = a.N; p.H = a.H; p.W = a.W;
     p.th = t.th; p.tw = t.tw; p.halo = t.halo; p.pitch = t.pitch; p.rows = t.rows;
     p.tiles_h = t.tiles_h; p.tiles_w = t.tiles_w; p.n_tiles = t.n_tiles;
-    int planes_max = 0, nmax = 0, cum = 0;
+    p.plane_bytes = t.rows_alloc * 128;
+    p.in_planes = planes_of(a.cin[0]);
+    p.in_bufs = t.in_bufs;
+    p.in_buf_bytes = p.in_planes * p.plane_bytes;
+    p.act_off = p.in_bufs * p.in_buf_bytes;
+    p.act_buf_bytes = t.act_planes * p.plane_bytes;
+    p.ring_off = p.act_off + t.act_bufs * p.act_buf_bytes;
+    p.stages = t.stages;
+    p.stage_bytes = t.stage_bytes;
+    p.bias_off = p.ring_off + p.stages * p.stage_bytes;
+    int cum = 0, boff = 0;
     for (int l = 0; l < a.n_layers; l++) {
         ChainLayerP& L = p.L[l];
         L.cin = a.cin[l]; L.cout = a.cout[l]; L.k = a.k[l]; L.pad = a.k[l] / 2; L.act = a.act[l];
-        L.n_pad = (a.cout[l] + 15) / 16 * 16;
-        L.slot = (L.n_pad + 31) / 32 * 32;
         L.kchunks = planes_of(a.cin[l]);
         L.ksteps_last = ((a.cin[l] - (L.kchunks - 1) * 64) + 15) / 16;
         cum += L.pad;
-        L.cum_pad = cum;
+        const LayerGeom g = layer_geom(a.cout[l], cum, t.rows, t.pitch);
+        L.qs = g.qs; L.range = g.range; L.nb = g.nb; L.n_pad = g.n_pad; L.n_chunks = g.n_chunks; L.chunk_n = g.chunk_n;
+        L.slot = g.slot; L.per_pass = g.per_pass;
+        L.bias_off = boff;
+        boff += g.n_pad;
         L.bias = a.bias[l];
-        planes_max = std::max(planes_max, std::max(planes_of(a.cin[l]), planes_of(L.n_pad)));
-        nmax = std::max(nmax, L.n_pad);
         const uint64_t taps = static_cast<uint64_t>(a.k[l]) * a.k[l];
         const uint64_t dims[3] = {static_cast<uint64_t>(a.cin[l]), taps, static_cast<uint64_t>(a.cout[l])};
         const uint64_t strides[2] = {static_cast<uint64_t>(a.cin[l]) * 2, taps * a.cin[l] * 2};
-        const uint32_t box[3] = {64, 1, static_cast<uint32_t>(L.n_pad)};
+        const uint32_t box[3] = {64, 1, static_cast<uint32_t>(std::min(g.chunk_n, g.n_pad))};
         const uint32_t es[3] = {1, 1, 1};
         int rc = encode_tmap(&p.tmw[l], a.w[l], 3, dims, strides, box, es);
         if (rc) return rc;
     }
-    const int rows_alloc = rows_alloc_of(a, t.rows, t.pitch);
-    p.plane_bytes = rows_alloc * 128;
-    p.buf_bytes = planes_max * p.plane_bytes;
-    p.in_planes = planes_of(a.cin[0]);
-    p.stages = t.stages;
-    p.stage_bytes = nmax * 128;
+    p.bias_floats = boff;
     p.pool = a.pool;
     p.base_offset_mode = base_offset_mode;
     p.cout_last = a.cout[a.n_layers - 1];

@@ -41,11 +41,16 @@ struct ChainTiling {
     int th, tw;          // output tile of the last layer (before pooling)
     int halo;            // sum of the layers' paddings
     int pitch, rows;     // frame of the input tile: (th + 2 halo) x (tw + 2 halo), pitch = width
+    int rows_alloc;      // rows one 64-channel plane holds (frame + reach of the last 128-row block)
     int tiles_h, tiles_w, n_tiles;
+    int in_bufs;         // 1 or 2 input frames resident (2 = next tile prefetched during compute)
+    int act_bufs;        // intermediate / staging buffers
+    int act_planes;
     int stages;          // weight ring depth
+    int stage_bytes;
     size_t smem_bytes;
-    int tmem_cols;
     double redundancy;   // computed / useful multiply-accumulates
+    double cost;         // the tiler's time estimate (arbitrary unit)
     bool ok;
 };
 
@@ -63,6 +68,7 @@ int launch_fc(const void* x, const void* w, const float* bias, void* y, int N, i
 
 // conv_tc.cu
 bool conv_tc_supported(const ConvArgs& a);
+bool chain_tc_layer_supported(int cin, int cout, int k);
 int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s);
 
 // chain_tc.cu

@@ -79,6 +79,12 @@ def test_single_layer(case):
     sess, xd, ref = _mk([layer], "single", n, h, w, layer["cin"])
     for s in (sms(), 3):
         G.check_plan(sess, xd, ref, [0], [s], "single S=%d" % s)
+    if layer["op"] == "conv" and layer["stride"] == 1 and layer["cin"] % 8 == 0:
+        # the same layer through the fused-chain kernel (input tile read once)
+        B.net_set_option(sess.net, B.OPT_SINGLE_AS_CHAIN, 1)
+        for s in (sms(), 3):
+            G.check_plan(sess, xd, ref, [0], [s], "single-as-chain S=%d" % s)
+        assert sess.kernels() == ["chain_tc"]
 
 
 def test_single_layer_with_residual_through_both_conv_kernels():
@@ -122,14 +128,17 @@ CHAINS = [
     (1, 56, 56, 32, (1, 1, 1, 1)),
     (3, 7, 7, 256, (3, 3)),
     (1, 28, 28, 64, (3, 3, 3, 3)),
+    (2, 28, 28, (128, 128, 512), (3, 1)),     # bottleneck tail: more than 256 output channels
+    (4, 14, 14, (128, 320, 64), (1, 3)),      # a wide intermediate map (5 planes, two channel chunks)
 ]
 
 
-@pytest.mark.parametrize("case", CHAINS, ids=lambda c: "%dx%dx%dx%d_%s" % (c[0], c[1], c[2], c[3], "".join(map(str, c[4]))))
+@pytest.mark.parametrize("case", CHAINS, ids=lambda c: "%dx%dx%dx%s_%s" % (c[0], c[1], c[2], c[3], "".join(map(str, c[4]))))
 def test_chain_every_contiguous_plan(case):
     n, h, w, c, ks = case
-    layers = [_conv(c, c, k, src=i - 1) for i, k in enumerate(ks)]
-    sess, xd, ref = _mk(layers, "chain", n, h, w, c)
+    cs = c if isinstance(c, tuple) else (c,) * (len(ks) + 1)
+    layers = [_conv(cs[i], cs[i + 1], k, src=i - 1) for i, k in enumerate(ks)]
+    sess, xd, ref = _mk(layers, "chain", n, h, w, cs[0])
     ran_fused = 0
     for ends in G.all_contiguous_plans(len(ks)):
         for s in (sms(), 5):
