@@ -188,8 +188,12 @@ const char* dlf_net_group_kernel(const dlf_net* net, int group);
  *                               only to document the measurement).
  *   DLF_OPT_SINGLE_AS_CHAIN  1: a single stride-1 1x1 / 3x3 convolution with <= 256 output
  *                               channels runs through the fused-chain kernel (input tile
- *                               loaded once) instead of the per-tap kernel. */
-enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3 };
+ *                               loaded once) instead of the per-tap kernel.
+ *   DLF_OPT_CUDA_GRAPH       1 (default): dlf_net_run replays one CUDA graph that holds every
+ *                               group of the plan (captured on the first run and whenever the
+ *                               input / output pointers, weights, workspace or plan change);
+ *                               0: launch the kernels one by one.  Does not clear the plan. */
+enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4 };
 int dlf_net_set_option(dlf_net* net, int option, int value);
 
 #ifdef __cplusplus

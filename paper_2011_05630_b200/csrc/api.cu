@@ -79,6 +79,16 @@ struct Group {
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+struct GraphCache {
+    cudaGraphExec_t exec = nullptr;
+    const void* in = nullptr;
+    void* out = nullptr;
+    void drop() {
+        if (exec) cudaGraphExecDestroy(exec);
+        exec = nullptr;
+    }
+};
+
 }  // namespace dlf
 
 using namespace dlf;
@@ -90,8 +100,14 @@ struct dlf_net {
     uint8_t* ws = nullptr;
     size_t ws_bytes = 0, ws_need = 0, in_off = 0, in_bytes = 0, status_off = 0;
     int dev_sms = 0;
-    int opt_no_tc = 0, opt_base_offset = 0, opt_single_chain = 0;
+    int opt_no_tc = 0, opt_base_offset = 0, opt_single_chain = 0, opt_graph = 1;
     const void* last_out = nullptr;
+    // One CUDA graph per (input, output) pointer pair holds the whole plan; a second, instrumented
+    // one records an event after every group for per-group timing.
+    dlf::GraphCache graph, graph_timed;
+    std::vector<cudaEvent_t> group_events;
+    cudaStream_t capture_stream = nullptr;
+    ~dlf_net();
 };
 
 namespace dlf {
@@ -264,6 +280,72 @@ static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* 
     return DLF_E_UNSUPPORTED;
 }
 
+}  // namespace dlf
+namespace dlf {
+int kernels_init() {
+    int rc = conv_tc_init();
+    return rc ? rc : chain_tc_init();
+}
+
+static void invalidate_graphs(dlf_net* net) {
+    net->graph.drop();
+    net->graph_timed.drop();
+}
+
+// Captures the launches of every group of the plan into one executable graph (thread-local
+// capture on a stream the net owns, so that nothing else the caller's thread or other threads
+// enqueue is swallowed).  With `timed`, an event is recorded before the first and after every group.
+static int build_graph(dlf_net* net, GraphCache* gc, const void* in_dev, void* out_dev, bool timed) {
+    gc->drop();
+    cudaError_t e;
+    if (!net->capture_stream) {
+        e = cudaStreamCreateWithFlags(&net->capture_stream, cudaStreamNonBlocking);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    if (timed) {
+        while (net->group_events.size() < net->plan.size() + 1) {
+            cudaEvent_t ev;
+            e = cudaEventCreate(&ev);
+            if (e != cudaSuccess) return cuda_fail(e);
+            net->group_events.push_back(ev);
+        }
+    }
+    cudaStream_t cs = net->capture_stream;
+    e = cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int rc = DLF_OK;
+    if (timed) cudaEventRecordWithFlags(net->group_events[0], cs, cudaEventRecordExternal);
+    for (size_t g = 0; g < net->plan.size() && rc == DLF_OK; g++) {
+        rc = launch_group(net, net->plan[g], in_dev, out_dev, cs);
+        if (timed && rc == DLF_OK) cudaEventRecordWithFlags(net->group_events[g + 1], cs, cudaEventRecordExternal);
+    }
+    cudaGraph_t graph = nullptr;
+    e = cudaStreamEndCapture(cs, &graph);
+    if (rc != DLF_OK) {
+        if (graph) cudaGraphDestroy(graph);
+        return rc;
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    e = cudaGraphInstantiate(&gc->exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) {
+        gc->exec = nullptr;
+        return cuda_fail(e);
+    }
+    gc->in = in_dev;
+    gc->out = out_dev;
+    return DLF_OK;
+}
+
+static int run_graph(dlf_net* net, GraphCache* gc, const void* in_dev, void* out_dev, bool timed, cudaStream_t s) {
+    if (!gc->exec || gc->in != in_dev || gc->out != out_dev) {
+        int rc = build_graph(net, gc, in_dev, out_dev, timed);
+        if (rc) return rc;
+    }
+    cudaError_t e = cudaGraphLaunch(gc->exec, s);
+    return e == cudaSuccess ? DLF_OK : cuda_fail(e);
+}
+
 static int check_ready(const dlf_net* net) {
     if (!net->ws) return DLF_E_WORKSPACE;
     if (net->plan.empty()) return DLF_E_STATE;
@@ -309,6 +391,13 @@ static int layer_sms(const Layer& l, const dlf_tuner_params& p, int s_max) {
 }
 
 }  // namespace dlf
+
+dlf_net::~dlf_net() {
+    graph.drop();
+    graph_timed.drop();
+    for (cudaEvent_t ev : group_events) cudaEventDestroy(ev);
+    if (capture_stream) cudaStreamDestroy(capture_stream);
+}
 
 // ---- C ABI ------------------------------------------------------------------------------------------
 
@@ -437,6 +526,7 @@ int dlf_net_set_weights(dlf_net* net, int layer, const void* w_f16_dev, const fl
     if (!is_param(l)) return DLF_E_INVALID_ARG;
     if ((reinterpret_cast<uintptr_t>(w_f16_dev) & 15) || (reinterpret_cast<uintptr_t>(bias_dev) & 15)) return DLF_E_INVALID_ARG;
     l.w = w_f16_dev;
+    invalidate_graphs(net);
     l.bias = bias_dev;
     return DLF_OK;
 }
@@ -455,6 +545,7 @@ int dlf_net_bind_workspace(dlf_net* net, void* workspace_dev, size_t bytes) {
         if (rc) return rc;
     }
     net->ws = static_cast<uint8_t*>(workspace_dev);
+    invalidate_graphs(net);
     net->ws_bytes = bytes;
     cudaError_t e = cudaMemset(net->ws + net->status_off, 0, 256);
     if (e != cudaSuccess) return cuda_fail(e);
@@ -471,6 +562,9 @@ int dlf_net_set_plan(dlf_net* net, int n_groups, const int32_t* group_end, const
     int rc = validate_plan(net, n_groups, group_end, sm_count, &plan);
     if (rc) return rc;
     net->plan.swap(plan);
+    invalidate_graphs(net);
+    rc = kernels_init();
+    if (rc) return rc;
     return DLF_OK;
 }
 
@@ -563,9 +657,14 @@ int dlf_net_run(dlf_net* net, const void* in_f16_dev, void* out_f16_dev, void* s
     int rc = check_ready(net);
     if (rc) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    for (const Group& g : net->plan) {
-        rc = launch_group(net, g, in_f16_dev, out_f16_dev, s);
+    if (net->opt_graph) {
+        rc = run_graph(net, &net->graph, in_f16_dev, out_f16_dev, false, s);
         if (rc) return rc;
+    } else {
+        for (const Group& g : net->plan) {
+            rc = launch_group(net, g, in_f16_dev, out_f16_dev, s);
+            if (rc) return rc;
+        }
     }
     net->last_out = out_f16_dev;
     return DLF_OK;
@@ -615,7 +714,7 @@ int dlf_net_time(dlf_net* net, const void* in_dev, void* out_dev, void* stream, 
     if (rc) return rc;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t ng = net->plan.size();
-    std::vector<cudaEvent_t> ev(ng + 1);
+    std::vector<cudaEvent_t> ev(2);
     for (auto& e : ev)
         if (cudaEventCreate(&e) != cudaSuccess) return cuda_fail(cudaGetLastError());
     auto cleanup = [&]() { for (auto& e : ev) cudaEventDestroy(e); };
@@ -640,20 +739,16 @@ int dlf_net_time(dlf_net* net, const void* in_dev, void* out_dev, void* stream, 
     if (ms_min) *ms_min = *std::min_element(times.begin(), times.end());
     if (ms_per_group) {
         std::vector<std::vector<float>> per(ng);
-        const int reps = std::min(iters, 20);
+        const int reps = std::min(std::max(iters, 3), 20);
         for (int i = 0; i < reps; i++) {
             if (flush_dev && flush_bytes) cudaMemsetAsync(flush_dev, i & 0xff, flush_bytes, s);
-            cudaEventRecord(ev[0], s);
-            for (size_t g = 0; g < ng; g++) {
-                rc = launch_group(net, net->plan[g], in_dev, out_dev, s);
-                if (rc) { cleanup(); return rc; }
-                cudaEventRecord(ev[g + 1], s);
-            }
-            cudaError_t e = cudaEventSynchronize(ev[ng]);
+            rc = run_graph(net, &net->graph_timed, in_dev, out_dev, true, s);
+            if (rc) { cleanup(); return rc; }
+            cudaError_t e = cudaStreamSynchronize(s);
             if (e != cudaSuccess) { cleanup(); return cuda_fail(e); }
             for (size_t g = 0; g < ng; g++) {
                 float ms = 0.0f;
-                cudaEventElapsedTime(&ms, ev[g], ev[g + 1]);
+                cudaEventElapsedTime(&ms, net->group_events[g], net->group_events[g + 1]);
                 per[g].push_back(ms);
             }
         }
@@ -694,17 +789,36 @@ int dlf_net_bruteforce(dlf_net* net, const dlf_search_params* sp, const void* in
                 if (S < 1 || S > net->dev_sms) continue;
                 Group g;
                 if (!make_group(net, a, a + len - 1, S, &g)) continue;
-                for (int i = 0; i < sp->warmup && rc == DLF_OK; i++) rc = launch_group(net, g, in_dev, final_out, s);
+                // a graph of kReps back-to-back launches hides the host's launch cost
+                const int kReps = 4;
+                cudaGraphExec_t exec = nullptr;
+                {
+                    if (!net->capture_stream && cudaStreamCreateWithFlags(&net->capture_stream, cudaStreamNonBlocking) != cudaSuccess)
+                        rc = cuda_fail(cudaGetLastError());
+                    cudaGraph_t graph = nullptr;
+                    if (rc == DLF_OK && cudaStreamBeginCapture(net->capture_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess)
+                        rc = cuda_fail(cudaGetLastError());
+                    if (rc == DLF_OK) {
+                        for (int r = 0; r < kReps && rc == DLF_OK; r++) rc = launch_group(net, g, in_dev, final_out, net->capture_stream);
+                        cudaError_t e = cudaStreamEndCapture(net->capture_stream, &graph);
+                        if (rc == DLF_OK && e != cudaSuccess) rc = cuda_fail(e);
+                        if (rc == DLF_OK && cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+                        if (graph) cudaGraphDestroy(graph);
+                    }
+                }
+                for (int i = 0; i < sp->warmup && rc == DLF_OK; i++)
+                    if (cudaGraphLaunch(exec, s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
                 std::vector<float> v;
                 for (int i = 0; i < sp->iters && rc == DLF_OK; i++) {
                     cudaEventRecord(e0, s);
-                    rc = launch_group(net, g, in_dev, final_out, s);
+                    if (cudaGraphLaunch(exec, s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
                     cudaEventRecord(e1, s);
                     if (cudaEventSynchronize(e1) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
                     float ms = 0.0f;
                     cudaEventElapsedTime(&ms, e0, e1);
-                    v.push_back(ms);
+                    v.push_back(ms / kReps);
                 }
+                if (exec) cudaGraphExecDestroy(exec);
                 if (rc == DLF_OK) {
                     const float m = median_of(v);
                     if (m < t[a][len - 1]) { t[a][len - 1] = m; ts[a][len - 1] = S; }
@@ -782,9 +896,11 @@ int dlf_net_set_option(dlf_net* net, int option, int value) {
         case DLF_OPT_NO_TENSOR_CORE: net->opt_no_tc = value != 0; break;
         case DLF_OPT_DESC_BASE_OFFSET: net->opt_base_offset = value != 0; break;
         case DLF_OPT_SINGLE_AS_CHAIN: net->opt_single_chain = value != 0; break;
+        case DLF_OPT_CUDA_GRAPH: net->opt_graph = value != 0; return DLF_OK;
         default: return DLF_E_INVALID_ARG;
     }
     net->plan.clear();  // kernel choices depend on the options: the plan must be set again
+    invalidate_graphs(net);
     return DLF_OK;
 }
 

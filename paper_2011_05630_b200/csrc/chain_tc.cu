@@ -495,11 +495,9 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
 int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int base_offset_mode, int* status_dev,
                     cudaStream_t s) {
     if (!t.ok) return DLF_E_PLAN;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return cuda_fail(e);
-        attr_set = true;
+    {
+        int rc = chain_tc_init();
+        if (rc) return rc;
     }
     ChainParams p;
     std::memset(&p, 0, sizeof(p));
@@ -560,6 +558,16 @@ int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int 
     chain_tc_kernel<<<grid, kThreads, smem, s>>>(p);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
+}
+
+int chain_tc_init() {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return cuda_fail(e);
+        attr_set = true;
+    }
+    return DLF_OK;
 }
 
 }  // namespace dlf

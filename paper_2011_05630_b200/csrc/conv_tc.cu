@@ -65,6 +65,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
+    if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 0);
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* stage0 = smem_raw + (base - smem_u32(smem_raw));
     const int stage_bytes = kABytes + p.BN * 128;
@@ -92,6 +93,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
     const int taps = p.kh * p.kw;
     const int k_iters = taps * p.kchunks;
@@ -115,6 +117,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                         tma_load_4d(sa, &tmx, &full_bar[st], kc * 64, c.wo0 * p.stride - p.pad + s,
                                     c.ho0 * p.stride - p.pad + r, c.n0);
                         tma_load_3d(sa + kABytes, &tmw, &full_bar[st], kc * 64, tap, c.co0);
+                        if (it == 0) DLF_TRACE_POINT(p.status, 2);
                     }
                 }
             }
@@ -135,6 +138,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     const int st = it % p.stages;
                     ok = mbar_wait(&full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                     if (!ok) break;
+                    if (it == 0) DLF_TRACE_POINT(p.status, 3);
                     tc_fence_after_sync();
                     const uint32_t sa = base + st * stage_bytes;
                     const int ksteps = ((ki % p.kchunks) == p.kchunks - 1) ? p.ksteps_last : 4;
@@ -145,6 +149,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     umma_commit(&empty_bar[st]);  // frees the stage once these MMAs have read it
                 }
                 if (ok) umma_commit(&tfull_bar[acc]);
+                if (j == 0) DLF_TRACE_POINT(p.status, 4);
             }
         }
     } else {
@@ -160,6 +165,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             const uint32_t acc = j & 1u;
             ok = mbar_wait(&tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
             if (!ok) break;
+            if (j == 0 && threadIdx.x == 64) DLF_TRACE_POINT(p.status, 5);
             tc_fence_after_sync();
             const int n = c.n0 + tn, ho = c.ho0 + th, wo = c.wo0 + tw;
             const bool valid = n < p.N && ho < p.Ho && wo < p.Wo;
@@ -215,6 +221,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+            if (j == 0 && threadIdx.x == 64) DLF_TRACE_POINT(p.status, 6);
         }
     }
 
@@ -224,6 +231,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         if (abort_s) __nanosleep(20000);  // let copies in flight land before the CTA retires
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, p.tmem_cols);
+        if (lane == 0) DLF_TRACE_POINT(p.status, 7);
     }
 }
 
@@ -262,11 +270,9 @@ bool conv_tc_supported(const ConvArgs& a) {
 
 int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s) {
     if (!conv_tc_supported(a)) return DLF_E_UNSUPPORTED;
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return cuda_fail(e);
-        attr_set = true;
+    {
+        int rc = conv_tc_init();
+        if (rc) return rc;
     }
     ConvTcParams p{};
     p.N = a.N; p.Ho = a.Ho; p.Wo = a.Wo; p.Cout = a.Cout;
@@ -321,6 +327,16 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     conv_tc_kernel<<<grid, kThreads, smem, s>>>(tmx, tmw, p);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
+}
+
+int conv_tc_init() {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return cuda_fail(e);
+        attr_set = true;
+    }
+    return DLF_OK;
 }
 
 }  // namespace dlf

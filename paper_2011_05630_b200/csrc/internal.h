@@ -57,6 +57,11 @@ struct ChainTiling {
 int cuda_fail(cudaError_t e);  // records the error for dlf_last_cuda_error, returns DLF_E_CUDA
 int cuda_fail_drv(int e);
 
+// Sets the kernels' shared-memory attributes once (outside any stream capture).
+int kernels_init();
+int conv_tc_init();
+int chain_tc_init();
+
 // kernels_mem.cu
 int launch_conv_direct(const ConvArgs& a, int sm_count, cudaStream_t s);
 int launch_dw3x3(const ConvArgs& a, int sm_count, cudaStream_t s);

@@ -19,6 +19,14 @@ __device__ __forceinline__ uint64_t global_ns() {
     return t;
 }
 
+// Optional timeline probe (compiled in only with -DDLF_TRACE): CTA 0 stores the global timer at
+// a few points after the status word.
+#ifdef DLF_TRACE
+#define DLF_TRACE_POINT(status, slot) do { if (blockIdx.x == 0) reinterpret_cast<volatile unsigned long long*>(status)[4 + (slot)] = global_ns(); } while (0)
+#else
+#define DLF_TRACE_POINT(status, slot) do { } while (0)
+#endif
+
 // ---- mbarrier ---------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
