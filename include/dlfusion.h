@@ -196,6 +196,41 @@ const char* dlf_net_group_kernel(const dlf_net* net, int group);
 enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4 };
 int dlf_net_set_option(dlf_net* net, int option, int value);
 
+/* Size of the scratch array that dlf_conv_chain_run_static keeps inside the library image. */
+#define DLF_STATIC_SCRATCH_BYTES (16u << 20)
+
+/* (The paper has no counterpart for this call.)
+ *
+ * Runs a chain of 1..8 dense convolutions (DLF_CONV, groups 1, no residual, no fused pool; layer i
+ * reads layer i-1, layer 0 reads x), one tensor-core kernel per layer, WITHOUT a workspace and
+ * without allocating anything: the maps between the layers and the kernels' status word live in
+ * a fixed DLF_STATIC_SCRATCH_BYTES (16 MiB) array that is part of the library and therefore
+ * occupies that much memory on every GPU that loads it, until the process exits.
+ *
+ * It is meant for callers that must not, or cannot, call cudaMalloc: code running between other
+ * frameworks that have already claimed the whole device, services with a fixed memory budget
+ * decided at start-up, and latency-critical loops in which an allocation's implicit device-wide
+ * synchronisation is unacceptable.  The caller still owns x, the weights, the biases and y.
+ *
+ *   layers[i].src must be i-1; cin, cout multiples of 8; stride 1 or 2.
+ *   w_f16_dev[i], bias_dev[i]: device pointers, layouts as for dlf_net_set_weights.
+ *   y_f16_dev: the last layer's output, fp16 NHWC.
+ *   sm_count: persistent grid size of every kernel (1 .. SMs of the device).
+ *
+ * Limits and errors: every map BETWEEN two layers must fit in half of the array (8 MiB), else
+ * DLF_E_WORKSPACE and nothing is enqueued; DLF_E_SHAPE / DLF_E_UNSUPPORTED / DLF_E_INVALID_ARG as
+ * for dlf_net_create.  The call enqueues on `stream`, waits for it, and returns DLF_E_TIMEOUT if
+ * a kernel's bounded wait gave up.
+ *
+ * The first call on a device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call before starting any stream capture.  All calls
+ * share the one array: it still holds the previous call's maps, the status word is cleared at
+ * the start of every call, and two calls that overlap on the same GPU (different streams or
+ * threads) overwrite each other's intermediate maps - run them one after another. */
+int dlf_conv_chain_run_static(const dlf_layer_desc* layers, int n_layers, int N, int H, int W,
+                              const void* x_f16_dev, const void* const* w_f16_dev,
+                              const float* const* bias_dev, void* y_f16_dev, int sm_count, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -74,6 +74,8 @@ def lib():
             "dlf_net_group_model": (C.c_int, [vp, C.c_int, i64p, i64p, C.POINTER(C.c_double), ip]),
             "dlf_net_group_kernel": (C.c_char_p, [vp, C.c_int]),
             "dlf_net_set_option": (C.c_int, [vp, C.c_int, C.c_int]),
+            "dlf_conv_chain_run_static": (C.c_int, [C.POINTER(LayerDesc), C.c_int, C.c_int, C.c_int, C.c_int, vp,
+                                                    C.POINTER(vp), C.POINTER(vp), vp, C.c_int, vp]),
         }
         for name, (res, args) in sig.items():
             f = getattr(L, name)
@@ -227,3 +229,16 @@ def net_group_kernel(net, g):
 
 def net_set_option(net, option, value):
     _check(lib().dlf_net_set_option(net, option, value), "dlf_net_set_option")
+
+
+STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def conv_chain_run_static(layers, n, h, w, x_ptr, w_ptrs, bias_ptrs, y_ptr, sm_count, stream=None):
+    """Chain of dense convolutions with the library's built-in scratch array (no workspace, no
+    allocation); waits for the stream.  Pointers are device addresses."""
+    arr = layers if isinstance(layers, C.Array) else layer_descs(layers)
+    wp = (C.c_void_p * len(arr))(*w_ptrs)
+    bp = (C.c_void_p * len(arr))(*bias_ptrs)
+    _check(lib().dlf_conv_chain_run_static(arr, len(arr), n, h, w, x_ptr, wp, bp, y_ptr, sm_count, stream),
+           "dlf_conv_chain_run_static")
