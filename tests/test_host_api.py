@@ -1,0 +1,140 @@
+"""Host-side logic of the library, without a GPU: the shared object loads and exports every
+symbol the header declares, layer lists are type-checked, operation counts and the auto-tuner
+(Eq. 5 + Algorithm 1) agree with the restated formulas in oracle/model.py."""
+import os
+import re
+
+import pytest
+
+from oracle import model
+from paper_2011_05630_b200 import binding as B, networks as nw
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    hdr = open(os.path.join(ROOT, "include", "dlfusion.h")).read()
+    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+    names = set(re.findall(r"\b(dlf_[a-z0-9_]+)\s*\(", hdr))
+    assert len(names) >= 24
+    lib = B.lib()
+    for n in sorted(names):
+        assert hasattr(lib, n), n
+    assert B.strerror(B.E_PLAN) == "invalid fusion plan" and B.strerror(0) == "ok"
+
+
+NETS = [("vgg16", nw.vgg16(), 8), ("resnet50", nw.resnet50(), 32), ("mobilenet_v2", nw.mobilenet_v2(), 64),
+        ("two_layer", nw.two_layer_group(), 1)]
+
+
+@pytest.mark.parametrize("name,layers,batch", NETS, ids=[n for n, _, _ in NETS])
+def test_shapes_and_operation_counts_match_the_formulas(name, layers, batch):
+    hw, c = (32, 16) if name == "two_layer" else (224, 3)
+    net = B.net_create(layers, batch, hw, hw, c)
+    shapes = model.infer_shapes(layers, batch, hw, hw, c)
+    lit = model.layer_ops(layers, batch, hw, hw, c, literal=True)
+    work = model.layer_ops(layers, batch, hw, hw, c, literal=False)
+    for i in range(len(layers)):
+        ops, fl, sh = B.net_layer_info(net, i)
+        assert sh == shapes[i], (i, sh, shapes[i])
+        assert ops == lit[i] and fl == work[i], (i, ops, lit[i], fl, work[i])
+    assert B.net_workspace_bytes(net) > sum(2 * s[0] * s[1] * s[2] * s[3] for s in shapes)
+    B.net_destroy(net)
+
+
+def _conv(cin, cout, k=3, **kw):
+    d = dict(op="conv", act="relu", cin=cin, cout=cout, kh=k, kw=k, stride=1, pad=k // 2, groups=1, src=-1, res_src=-2, pool=0)
+    d.update(kw)
+    return d
+
+
+@pytest.mark.parametrize("layers,status", [
+    ([_conv(8, 8), _conv(16, 8, src=0)], B.E_SHAPE),            # channel mismatch
+    ([_conv(8, 8, src=0)], B.E_SHAPE),                            # reads itself
+    ([_conv(8, 8, kh=9, kw=9, pad=0)], B.E_SHAPE),                # kernel larger than the image
+    ([_conv(8, 8), _conv(8, 16, src=0, res_src=-1)], B.E_SHAPE),  # residual of another shape
+    ([_conv(8, 8, groups=3)], B.E_SHAPE),
+    ([_conv(8, 8, stride=0)], B.E_INVALID_ARG),
+    ([_conv(8, 8, pool=3)], B.E_INVALID_ARG),
+    ([dict(_conv(8, 8), op="fc", cin=7)], B.E_SHAPE),
+    ([_conv(8, 12, groups=4)], B.E_UNSUPPORTED),                  # grouped conv without a kernel
+    ([dict(_conv(12, 12, groups=12), op="dwconv")], B.E_UNSUPPORTED),
+])
+def test_bad_layer_lists_are_rejected(layers, status):
+    with pytest.raises(B.DlfError) as e:
+        B.net_create(layers, 1, 6, 6, layers[0]["cin"])
+    assert e.value.status == status
+
+
+def test_bad_arguments_and_call_order():
+    import ctypes as C
+    L = B.lib()
+    assert L.dlf_net_create(None, 1, 1, 4, 4, 8, C.byref(C.c_void_p())) == B.E_INVALID_ARG
+    arr = B.layer_descs([_conv(8, 8)])
+    assert L.dlf_net_create(arr, 0, 1, 4, 4, 8, C.byref(C.c_void_p())) == B.E_INVALID_ARG
+    assert L.dlf_net_create(arr, 1, 0, 4, 4, 8, C.byref(C.c_void_p())) == B.E_INVALID_ARG
+    net = B.net_create([_conv(8, 8)], 1, 4, 4, 8)
+    assert L.dlf_net_run(net, 256, 512, None) == B.E_WORKSPACE          # nothing bound yet
+    assert L.dlf_net_bind_workspace(net, 256, 16) == B.E_WORKSPACE      # too small
+    assert L.dlf_net_bind_workspace(net, 300, 1 << 30) == B.E_WORKSPACE  # misaligned
+    assert L.dlf_net_set_weights(net, 0, None, None) == B.E_INVALID_ARG
+    assert L.dlf_net_set_weights(net, 5, 256, 256) == B.E_INVALID_ARG
+    assert L.dlf_net_set_weights(net, 0, 264, 256) == B.E_INVALID_ARG    # not 16-byte aligned
+    assert L.dlf_net_layer_info(net, 3, None, None, None) == B.E_INVALID_ARG
+    assert L.dlf_net_set_option(net, 99, 1) == B.E_INVALID_ARG
+    assert L.dlf_net_boundary_tensor(net, 0, C.byref(C.c_void_p()), None) == B.E_WORKSPACE
+    assert L.dlf_conv_chain_run_static(arr, 0, 1, 4, 4, 256, None, None, 256, 1, None) == B.E_INVALID_ARG
+    B.net_destroy(net)
+
+
+# ---- the auto-tuner against the restated Algorithm 1 ----------------------------------------------------
+def _chain_layer_ok(l):
+    return (l["op"] == "conv" and l["groups"] == 1 and l["stride"] == 1 and l["kh"] == l["kw"] and l["kh"] in (1, 3)
+            and l["pad"] == l["kh"] // 2 and l["cin"] % 8 == 0 and l["cout"] % 8 == 0 and 8 <= l["cin"] <= 1024
+            and 8 <= l["cout"] <= 2048)
+
+
+def span_is_chain(layers, first, last):
+    """The structural rule of fusable spans, written from its description: a chain of dense
+    stride-1 size-keeping 1x1/3x3 convolutions, each reading its predecessor, pool / residual on
+    the last layer only, no intermediate map used anywhere else; at most 8 layers."""
+    if last - first + 1 > 8:
+        return False
+    for i in range(first, last + 1):
+        l = layers[i]
+        if not _chain_layer_ok(l):
+            return False
+        if i > first and l["src"] != i - 1:
+            return False
+        if i < last and (l["pool"] != 0 or l["res_src"] != -2):
+            return False
+        if i == last and l["res_src"] >= first:
+            return False
+    inter = set(range(first, last))
+    for j in range(first + 1, len(layers)):
+        l = layers[j]
+        for which, r in (("src", l["src"]), ("res", l["res_src"])):
+            if r in inter and not (which == "src" and j <= last and r == j - 1 and l["res_src"] != r):
+                return False
+    return True
+
+
+P = dict(alpha=0.316, beta=0.659, kappa=12.0, kappa0=-170.0, s_max=148)
+
+
+@pytest.mark.parametrize("name,layers,batch", NETS + [("chain8", nw.conv_chain(8, 64, 3), 16),
+                                                     ("chain_1x1", nw.conv_chain(6, 128, 1), 8)],
+                         ids=[n for n, _, _ in NETS] + ["chain8", "chain_1x1"])
+@pytest.mark.parametrize("crit", [1.0, 1e7, 2e8, 3e9, 1e11, 1e30])
+def test_autotune_equals_restated_algorithm1(name, layers, batch, crit):
+    hw, c = {"two_layer": (32, 16), "chain8": (56, 64), "chain_1x1": (28, 128)}.get(name, (224, 3))
+    net = B.net_create(layers, batch, hw, hw, c)
+    ops = model.layer_ops(layers, batch, hw, hw, c)
+    kinds = [l["op"] in ("conv", "dwconv", "fc") for l in layers]
+    ch = [l["cout"] for l in layers]
+    n = len(layers)
+    want = model.algorithm1(kinds, ch, ops, dict(P, op_critical=crit),
+                            must_close_after=lambda start, i: i == n - 1 or not span_is_chain(layers, start, i + 1))
+    got = B.net_autotune(net, n, P["alpha"], P["beta"], P["kappa"], P["kappa0"], crit, s_max=148, legalise=0)
+    assert got == (want[0], want[1]), (got, want)
+    B.net_destroy(net)
