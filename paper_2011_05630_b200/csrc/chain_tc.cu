@@ -21,8 +21,9 @@
 // global memory.  Weights stream through a TMA ring, once per pass; the next tile's input frame
 // is prefetched into a second buffer while the current tile computes.
 //
-// Warp roles: 0 weight producer, 1 UMMA issuer (owns the TMEM allocation), 2-5 epilogue,
-// 6 input producer.
+// Warp roles: 0 weight producer, 1 UMMA issuer (owns the TMEM allocation), 2-9 epilogue (two per
+// TMEM lane quarter, alternating 32-column chunks), 10 input producer.  The epilogue is
+// specialised at compile time on (activation, destination): see epi_pass.
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -37,7 +38,9 @@ namespace dlf {
 
 namespace {
 
-constexpr int kThreads = 224;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps + 32;
+constexpr int kInputWarp = 2 + kEpiWarps;
 constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
 constexpr int kMaxBias = 4096;           // floats of bias staged in shared memory (all layers)
 
@@ -72,10 +75,88 @@ struct ChainParams {
     int* status;
 };
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory"); }
 
 __device__ __forceinline__ int chunk_cols(const ChainLayerP& L, int c) {
     return min(L.chunk_n, L.n_pad - c * L.chunk_n);
+}
+
+struct EpiCtx {
+    int row, half;            // TMEM lane of this thread; which alternating 32-column chunks it takes
+    uint32_t tmem_lane, tmem_col;
+    int gy0, gx0, n;          // image coordinates of frame row 0 / column 0, image index
+    int b0, nblk, ncols, ch0; // blocks of this pass, columns and first channel of this chunk
+    uint8_t* obuf;
+    const float* bl;
+    float act_lo, act_hi;
+};
+
+// Drains one pass.  MODE 0: next layer's operand tile in shared memory (zero outside the image);
+// 1: global memory; 2: global memory with residual; 3: shared staging tile with residual (pooled
+// last layer).  The activation is a clamp to [act_lo, act_hi] (none: -inf..inf, ReLU: 0..inf,
+// ReLU6: 0..6), which keeps the loop free of branches without one copy of the code per activation.
+template <int MODE>
+__device__ __forceinline__ void epi_pass(const ChainParams& p, const ChainLayerP& L, const EpiCtx& cx) {
+    constexpr bool kGlobal = (MODE == 1 || MODE == 2);
+    constexpr bool kRes = (MODE == 2 || MODE == 3);
+    for (int b = 0; b < cx.nblk; b++) {
+        const int q = L.qs + (cx.b0 + b) * 128 + cx.row;
+        const int fy = q / p.pitch, fx = q - fy * p.pitch;
+        const int gy = cx.gy0 + fy, gx = cx.gx0 + fx;
+        const bool in_img = gy >= 0 && gy < p.H && gx >= 0 && gx < p.W;
+        const bool in_tile = fy >= p.halo && fy < p.halo + p.th && fx >= p.halo && fx < p.halo + p.tw;
+        const bool live = q < L.qs + L.range && (!kGlobal || (in_img && in_tile));
+        const long long gpix = (static_cast<long long>(cx.n) * p.H + gy) * p.W + gx;
+        const uint32_t taddr = cx.tmem_lane + cx.tmem_col + b * L.slot;
+        for (int cc = cx.half * 32; cc < cx.ncols; cc += 64) {
+            float v[32];
+            __syncwarp();  // the aligned TMEM loads need the whole warp converged
+            const int nc = min(32, cx.ncols - cc);
+            if (nc == 32) tmem_ld32(taddr + cc, v);
+            else tmem_ld16(taddr + cc, v);
+            if (!live) continue;
+#pragma unroll
+            for (int g = 0; g < 4; g++) {
+                if (g * 8 >= nc) break;
+                const int co = cx.ch0 + cc + g * 8;  // first of 8 channels
+                uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                if (kGlobal || in_img) {
+                    float a[8];
+                    const float4 b0 = *reinterpret_cast<const float4*>(cx.bl + co);
+                    const float4 b1 = *reinterpret_cast<const float4*>(cx.bl + co + 4);
+                    a[0] = v[g * 8 + 0] + b0.x; a[1] = v[g * 8 + 1] + b0.y; a[2] = v[g * 8 + 2] + b0.z; a[3] = v[g * 8 + 3] + b0.w;
+                    a[4] = v[g * 8 + 4] + b1.x; a[5] = v[g * 8 + 5] + b1.y; a[6] = v[g * 8 + 6] + b1.z; a[7] = v[g * 8 + 7] + b1.w;
+                    if (kRes) {
+                        if (co < L.cout && (kGlobal || in_tile)) {
+                            const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.res + gpix * L.cout + co));
+                            const __half2* rh = reinterpret_cast<const __half2*>(&rv);
+#pragma unroll
+                            for (int e = 0; e < 4; e++) {
+                                const float2 rf = __half22float2(rh[e]);
+                                a[2 * e] += rf.x;
+                                a[2 * e + 1] += rf.y;
+                            }
+                        }
+                    }
+                    // channels past cout (padding up to 16) carry zero weights and zero bias: act(0) = 0,
+                    // so the next layer's K padding stays zero
+#pragma unroll
+                    for (int e = 0; e < 8; e++) a[e] = fminf(fmaxf(a[e], cx.act_lo), cx.act_hi);
+                    val.x = pack_half2(a[0], a[1]);
+                    val.y = pack_half2(a[2], a[3]);
+                    val.z = pack_half2(a[4], a[5]);
+                    val.w = pack_half2(a[6], a[7]);
+                }
+                if (kGlobal) {
+                    if (co < L.cout) *reinterpret_cast<uint4*>(p.out + gpix * L.cout + co) = val;
+                } else {
+                    const int g8 = co >> 3;  // 8-channel group index
+                    *reinterpret_cast<uint4*>(cx.obuf + static_cast<size_t>(g8 >> 3) * p.plane_bytes + static_cast<size_t>(q) * 128 +
+                                              (((g8 & 7) ^ (q & 7)) << 4)) = val;
+                }
+            }
+        }
+    }
 }
 
 __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainParams p) {
@@ -101,9 +182,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             mbar_init(&in_full_bar[i], 1);
             mbar_init(&in_empty_bar[i], 1);
             mbar_init(&acc_full_bar[i], 1);
-            mbar_init(&acc_empty_bar[i], 4);
+            mbar_init(&acc_empty_bar[i], kEpiWarps);
         }
-        mbar_init(&act_ready_bar, 4);
+        mbar_init(&act_ready_bar, kEpiWarps);
         fence_barrier_init();
         tma_prefetch_desc(&p.tmx);
     }
@@ -121,7 +202,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     const uint32_t tmem_base = tmem_base_s;
     const int frame_rows = p.rows * p.pitch;
 
-    if (warp == 6) {
+    if (warp == kInputWarp) {
         // ---- input producer: one frame per tile, prefetched into the free input buffer ---------
         if (lane == 0) {
             uint32_t tile_i = 0;
@@ -196,15 +277,19 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                                                    0x600 | (blockIdx.x << 12));
                                     if (!ok) break;
                                     tc_fence_after_sync();
-                                    const uint32_t wsm = base + p.ring_off + st * p.stage_bytes;
+                                    const uint32_t b_lo = umma_desc_lo(base + p.ring_off + st * p.stage_bytes);
                                     const int ksteps = (kc == L.kchunks - 1) ? L.ksteps_last : 4;
-                                    for (int b = 0; b < nblk; b++) {
-                                        const uint32_t arow = abuf + kc * p.plane_bytes + (L.qs + (b0 + b) * 128 + shift) * 128;
-                                        const uint32_t bo = p.base_offset_mode ? ((arow >> 7) & 7u) : 0u;
-                                        const uint32_t d_tmem = tmem_base + half * 256u + b * L.slot;
-                                        for (int ks = 0; ks < ksteps; ks++)
-                                            umma_f16(d_tmem, umma_desc_sw128(arow + ks * 32, bo),
-                                                     umma_desc_sw128(wsm + ks * 32, 0), idesc, (tap | kc | ks) != 0);
+                                    const uint32_t arow0 = abuf + kc * p.plane_bytes + (L.qs + b0 * 128 + shift) * 128;
+                                    const uint32_t acc0 = (tap | kc) != 0;
+                                    uint32_t d_tmem = tmem_base + half * 256u;
+                                    for (int b = 0; b < nblk; b++, d_tmem += L.slot) {
+                                        const uint32_t arow = arow0 + b * (128 * 128);
+                                        const uint32_t a_lo = umma_desc_lo(arow);
+                                        const uint32_t a_hi = p.base_offset_mode ? (kDescHiSw128 | (((arow >> 7) & 7u) << 17)) : kDescHiSw128;
+                                        umma_f16_lo(d_tmem, a_lo, a_hi, b_lo, idesc, acc0);
+                                        if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, a_hi, b_lo + 2, idesc, 1);
+                                        if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, a_hi, b_lo + 4, idesc, 1);
+                                        if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, a_hi, b_lo + 6, idesc, 1);
                                     }
                                     umma_commit(&wempty_bar[st]);
                                 }
@@ -218,98 +303,43 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             }
         }
     } else {
-        // ---- epilogue warps (128 threads = 128 TMEM lanes) -------------------------------------------------
-        const int q4 = warp & 3;
-        const int row = q4 * 32 + lane;
-        const int et = threadIdx.x - 64;  // 0..127
+        // ---- epilogue warps ------------------------------------------------------------------------------------
+        const int et = threadIdx.x - 64;  // 0 .. 32*kEpiWarps-1
+        EpiCtx cx;
+        cx.row = (warp & 3) * 32 + lane;
+        cx.half = (warp - 2) >> 2;
+        cx.tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         uint32_t pass_i = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
             const int txi = t % p.tiles_w, tyi = (t / p.tiles_w) % p.tiles_h, n = t / (p.tiles_w * p.tiles_h);
-            const int gy0 = tyi * p.th - p.halo, gx0 = txi * p.tw - p.halo;
+            cx.gy0 = tyi * p.th - p.halo;
+            cx.gx0 = txi * p.tw - p.halo;
+            cx.n = n;
             for (int l = 0; l < p.n_layers && ok; l++) {
                 const ChainLayerP& L = p.L[l];
                 const bool last = (l == p.n_layers - 1);
-                const bool to_global = last && !p.pool;
-                uint8_t* obuf = sbase + p.act_off + (l & 1) * p.act_buf_bytes;
-                const float* bl = bias_s + L.bias_off;
+                const int mode = (last && !p.pool) ? (p.res != nullptr ? 2 : 1) : ((last && p.res != nullptr) ? 3 : 0);
+                cx.obuf = sbase + p.act_off + (l & 1) * p.act_buf_bytes;
+                cx.bl = bias_s + L.bias_off;
+                cx.act_lo = L.act >= 1 ? 0.0f : -INFINITY;
+                cx.act_hi = L.act == 2 ? 6.0f : INFINITY;
                 for (int c = 0; c < L.n_chunks && ok; c++) {
-                    const int ncols = chunk_cols(L, c), ch0 = c * L.chunk_n;
+                    cx.ncols = chunk_cols(L, c);
+                    cx.ch0 = c * L.chunk_n;
                     for (int b0 = 0; b0 < L.nb && ok; b0 += L.per_pass, pass_i++) {
-                        const int nblk = min(L.per_pass, L.nb - b0);
                         const uint32_t half = pass_i & 1u;
                         ok = mbar_wait(&acc_full_bar[half], (pass_i >> 1) & 1u, abort_flag, p.status, 0x700 | (blockIdx.x << 12));
                         if (!ok) break;
                         tc_fence_after_sync();
-                        for (int b = 0; b < nblk; b++) {
-                            const int q = L.qs + (b0 + b) * 128 + row;
-                            const int fy = q / p.pitch, fx = q - fy * p.pitch;
-                            const int gy = gy0 + fy, gx = gx0 + fx;
-                            const bool in_range = q < L.qs + L.range;
-                            const bool in_img = gy >= 0 && gy < p.H && gx >= 0 && gx < p.W;
-                            const bool in_tile = fy >= p.halo && fy < p.halo + p.th && fx >= p.halo && fx < p.halo + p.tw;
-                            const long long gpix = (static_cast<long long>(n) * p.H + gy) * p.W + gx;
-                            const bool live = in_range && (to_global ? (in_img && in_tile) : true);
-                            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16) + half * 256u + b * L.slot;
-                            for (int cc = 0; cc < ncols; cc += 32) {
-                                float v[32];
-                                __syncwarp();  // the aligned TMEM loads need the whole warp converged
-                                const int nc = min(32, ncols - cc);
-                                if (nc == 32) tmem_ld32(taddr + cc, v);
-                                else tmem_ld16(taddr + cc, v);
-                                if (!live) continue;
-                                for (int h = 0; h < nc; h += 16) {
-                                    const int co = ch0 + cc + h;  // first of 16 channels
-                                    uint32_t packed[8];
-                                    if (in_img) {
-                                        float a[16];
-#pragma unroll
-                                        for (int e = 0; e < 16; e += 4) {
-                                            const float4 bb = *reinterpret_cast<const float4*>(bl + co + e);
-                                            a[e] = v[h + e] + bb.x; a[e + 1] = v[h + e + 1] + bb.y;
-                                            a[e + 2] = v[h + e + 2] + bb.z; a[e + 3] = v[h + e + 3] + bb.w;
-                                        }
-                                        if (last && p.res != nullptr) {
-#pragma unroll
-                                            for (int g = 0; g < 2; g++) {
-                                                if (co + g * 8 < L.cout) {
-                                                    const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.res + gpix * L.cout + co + g * 8));
-                                                    const __half2* rh = reinterpret_cast<const __half2*>(&rv);
-#pragma unroll
-                                                    for (int e = 0; e < 4; e++) {
-                                                        const float2 rf = __half22float2(rh[e]);
-                                                        a[g * 8 + 2 * e] += rf.x;
-                                                        a[g * 8 + 2 * e + 1] += rf.y;
-                                                    }
-                                                }
-                                            }
-                                        }
-#pragma unroll
-                                        for (int e = 0; e < 8; e++)
-                                            packed[e] = pack_half2(apply_act(a[2 * e], L.act), apply_act(a[2 * e + 1], L.act));
-                                        // channels past cout (padding up to 16) carry zero weights and zero bias:
-                                        // act(0) = 0, so the next layer's K padding stays zero
-                                    } else {
-#pragma unroll
-                                        for (int e = 0; e < 8; e++) packed[e] = 0u;
-                                    }
-#pragma unroll
-                                    for (int g = 0; g < 2; g++) {
-                                        const uint4 val = make_uint4(packed[g * 4], packed[g * 4 + 1], packed[g * 4 + 2], packed[g * 4 + 3]);
-                                        if (to_global) {
-                                            if (co + g * 8 < L.cout)
-                                                *reinterpret_cast<uint4*>(p.out + gpix * L.cout + co + g * 8) = val;
-                                        } else {
-                                            const int g8 = (co >> 3) + g;  // 8-channel group index
-                                            uint8_t* dst = obuf + static_cast<size_t>(g8 >> 3) * p.plane_bytes +
-                                                           static_cast<size_t>(q) * 128 + (((g8 & 7) ^ (q & 7)) << 4);
-                                            *reinterpret_cast<uint4*>(dst) = val;
-                                        }
-                                    }
-                                }
-                            }
-                        }
-                        if (!to_global) fence_proxy_async_smem();  // UMMA reads these rows through the async proxy
+                        cx.b0 = b0;
+                        cx.nblk = min(L.per_pass, L.nb - b0);
+                        cx.tmem_col = half * 256u;
+                        if (mode == 0) epi_pass<0>(p, L, cx);
+                        else if (mode == 1) epi_pass<1>(p, L, cx);
+                        else if (mode == 2) epi_pass<2>(p, L, cx);
+                        else epi_pass<3>(p, L, cx);
+                        if (mode == 0 || mode == 3) fence_proxy_async_smem();  // UMMA reads these rows through the async proxy
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&acc_empty_bar[half]);
@@ -326,7 +356,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                 const int oth = p.th / 2, otw = p.tw / 2;
                 const int Ho = p.H / 2, Wo = p.W / 2;
                 const int total = oth * otw * c8n;
-                for (int i = et; i < total; i += 128) {
+                for (int i = et; i < total; i += 32 * kEpiWarps) {
                     const int g8 = i % c8n;
                     const int ox = (i / c8n) % otw, oy = i / (c8n * otw);
                     const int gy = tyi * oth + oy, gx = txi * otw + ox;

@@ -1,5 +1,5 @@
-// Single-layer implicit-GEMM convolution on the tcgen05 tensor cores (the kernel of the
-// no-fusion plan, and of every group that holds one dense convolution).
+// Single-layer implicit-GEMM convolution on the tcgen05 tensor cores (general stride; the
+// kernel of every group that holds one dense convolution the fused-chain kernel does not take).
 //
 //   D[m, n] = sum over (tap, ci) of A_tap[m, ci] * W[n, tap, ci]        (Eq. 1 counts these MACs)
 //   M = 128 output pixels (a TN x TH x TW patch), N = up to 256 output channels, K = taps x C_in.
@@ -8,9 +8,13 @@
 // work list.  Per CTA: one producer thread issues TMA tiled loads (the tap's shifted, strided
 // window of the NHWC input, zero-filled outside the image = the convolution's padding; and the
 // tap's [C_out][64] weight slab) into a ring of 128-byte-swizzled stages; one thread issues
-// tcgen05.mma (fp16 x fp16 -> fp32) into one of two TMEM accumulators; four epilogue warps read
-// the other accumulator with tcgen05.ld and apply bias, residual, activation, the fp16 rounding
-// and the optional 2x2 max-pool (warp shuffles) before 16-byte global stores.
+// tcgen05.mma (fp16 x fp16 -> fp32) into one of two TMEM accumulators; eight epilogue warps (two
+// per TMEM lane quarter, alternating 32-column chunks) drain the other accumulator: bias (staged
+// in shared memory), residual, activation, fp16 rounding.  Without pooling the tile is written to
+// a swizzled staging buffer and leaves through TMA stores (clipped at the tensor's edges); with
+// the fused 2x2 max-pool the window is reduced by warp shuffles and written with 16-byte stores.
+// The epilogue is specialised at compile time on (activation, pool, residual): it is the part of
+// the kernel that bounds memory-bound layers, and runtime branches there cost more than the math.
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -23,7 +27,8 @@ namespace dlf {
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr int kABytes = 128 * 128;  // 128 pixels x 64 fp16
 constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
 
@@ -33,8 +38,9 @@ struct ConvTcParams {
     int TW, TH, TN, tiles_w, tiles_h, tiles_n;
     int BN, n_tiles_n, acc_stride;
     int kchunks, ksteps_last;
-    int act, pool, stages;
+    int stages;
     int n_work;
+    int stage_out_off, bias_off;  // byte offsets in dynamic shared memory
     uint32_t tmem_cols;
     const float* bias;
     const __half* res;
@@ -58,8 +64,12 @@ __device__ __forceinline__ TileCoord decode_work(const ConvTcParams& p, int t) {
     return c;
 }
 
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory"); }
+
+template <int ACT, bool POOL, bool RES>
 __global__ void __launch_bounds__(kThreads, 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw, const ConvTcParams p) {
+conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
+               const __grid_constant__ CUtensorMap tmy, const ConvTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[8], empty_bar[8], tfull_bar[2], tempty_bar[2];
     __shared__ uint32_t tmem_base_s;
@@ -68,6 +78,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 0);
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* stage0 = smem_raw + (base - smem_u32(smem_raw));
+    float* bias_s = reinterpret_cast<float*>(stage0 + p.bias_off);
     const int stage_bytes = kABytes + p.BN * 128;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &abort_s;
@@ -80,15 +91,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         }
         for (int i = 0; i < 2; i++) {
             mbar_init(&tfull_bar[i], 1);
-            mbar_init(&tempty_bar[i], 4);
+            mbar_init(&tempty_bar[i], kEpiWarps);
         }
         fence_barrier_init();
         tma_prefetch_desc(&tmx);
         tma_prefetch_desc(&tmw);
+        if (!POOL) tma_prefetch_desc(&tmy);
     }
     if (warp == 1) {
         tmem_alloc(&tmem_base_s, p.tmem_cols);
         tmem_relinquish();
+    }
+    {   // bias of every output channel, zero past C_out (the channel tile is padded to 16)
+        const int n_bias = p.n_tiles_n * p.BN;
+        for (int i = threadIdx.x; i < n_bias; i += kThreads) bias_s[i] = i < p.Cout ? __ldg(p.bias + i) : 0.0f;
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -134,19 +150,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * p.acc_stride;
+                int kc = 0;
                 for (int ki = 0; ki < k_iters; ki++, it++) {
                     const int st = it % p.stages;
                     ok = mbar_wait(&full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                     if (!ok) break;
                     if (it == 0) DLF_TRACE_POINT(p.status, 3);
                     tc_fence_after_sync();
-                    const uint32_t sa = base + st * stage_bytes;
-                    const int ksteps = ((ki % p.kchunks) == p.kchunks - 1) ? p.ksteps_last : 4;
-                    for (int ks = 0; ks < ksteps; ks++) {
-                        umma_f16(d_tmem, umma_desc_sw128(sa + ks * 32, 0), umma_desc_sw128(sa + kABytes + ks * 32, 0),
-                                 idesc, (ki | ks) != 0);
-                    }
+                    const uint32_t a_lo = umma_desc_lo(base + st * stage_bytes), b_lo = umma_desc_lo(base + st * stage_bytes + kABytes);
+                    const int ksteps = (kc == p.kchunks - 1) ? p.ksteps_last : 4;
+                    umma_f16_lo(d_tmem, a_lo, kDescHiSw128, b_lo, idesc, ki != 0);
+                    if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, kDescHiSw128, b_lo + 2, idesc, 1);
+                    if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, kDescHiSw128, b_lo + 4, idesc, 1);
+                    if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, kDescHiSw128, b_lo + 6, idesc, 1);
                     umma_commit(&empty_bar[st]);  // frees the stage once these MMAs have read it
+                    if (++kc == p.kchunks) kc = 0;
                 }
                 if (ok) umma_commit(&tfull_bar[acc]);
                 if (j == 0) DLF_TRACE_POINT(p.status, 4);
@@ -154,10 +172,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         }
     } else {
         // ---- epilogue warps ---------------------------------------------------------------------------
-        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        const int q = warp & 3;              // TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;    // which of the alternating 32-column chunks
         const int m = q * 32 + lane;
         const int tw = m % p.TW, th = (m / p.TW) % p.TH, tn = m / (p.TW * p.TH);
-        const int Hp = p.pool ? p.Ho / 2 : p.Ho, Wp = p.pool ? p.Wo / 2 : p.Wo;
+        const int Hp = POOL ? p.Ho / 2 : p.Ho, Wp = POOL ? p.Wo / 2 : p.Wo;
+        uint8_t* stage_out = stage0 + p.stage_out_off;
+        const bool issuer = (threadIdx.x == 64);
         uint32_t j = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
@@ -165,64 +186,78 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             const uint32_t acc = j & 1u;
             ok = mbar_wait(&tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
             if (!ok) break;
-            if (j == 0 && threadIdx.x == 64) DLF_TRACE_POINT(p.status, 5);
+            if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 5);
             tc_fence_after_sync();
             const int n = c.n0 + tn, ho = c.ho0 + th, wo = c.wo0 + tw;
             const bool valid = n < p.N && ho < p.Ho && wo < p.Wo;
             const long long pix = (static_cast<long long>(n) * p.Ho + ho) * p.Wo + wo;
-            const long long opix = p.pool ? (static_cast<long long>(n) * Hp + (ho >> 1)) * Wp + (wo >> 1) : pix;
-            const bool writer = valid && (!p.pool || (((ho | wo) & 1) == 0 && (ho >> 1) < Hp && (wo >> 1) < Wp));
+            const long long opix = POOL ? (static_cast<long long>(n) * Hp + (ho >> 1)) * Wp + (wo >> 1) : pix;
+            const bool writer = valid && (!POOL || (((ho | wo) & 1) == 0 && (ho >> 1) < Hp && (wo >> 1) < Wp));
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.acc_stride;
-            const int ncols = min(p.BN, p.Cout - c.co0);
-            for (int cc = 0; cc < ncols; cc += 16) {
-                float v[16];
+            const int ncols = min(p.BN, ((p.Cout - c.co0) + 15) & ~15);
+            for (int cc = half * 32; cc < ncols; cc += 64) {
+                float v[32];
                 __syncwarp();  // the aligned TMEM load needs the whole warp converged
-                tmem_ld16(taddr + cc, v);
-                const int co = c.co0 + cc;
-                const int nv = min(16, p.Cout - co);  // 8 or 16
+                const int nc = min(32, ncols - cc);
+                if (nc == 32) tmem_ld32(taddr + cc, v);
+                else tmem_ld16(taddr + cc, v);
 #pragma unroll
-                for (int h8 = 0; h8 < 2; h8++) {
-                    if (h8 * 8 >= nv) break;
-                    const float4 b0 = __ldg(reinterpret_cast<const float4*>(p.bias + co + h8 * 8));
-                    const float4 b1 = __ldg(reinterpret_cast<const float4*>(p.bias + co + h8 * 8 + 4));
-                    float* vv = v + h8 * 8;
-                    vv[0] += b0.x; vv[1] += b0.y; vv[2] += b0.z; vv[3] += b0.w;
-                    vv[4] += b1.x; vv[5] += b1.y; vv[6] += b1.z; vv[7] += b1.w;
-                    if (p.res != nullptr && valid) {
-                        const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.res + pix * p.Cout + co + h8 * 8));
-                        const __half2* rh = reinterpret_cast<const __half2*>(&rv);
+                for (int g = 0; g < 4; g++) {
+                    if (g * 8 >= nc) break;
+                    const int co = c.co0 + cc + g * 8;  // first of 8 channels
+                    float a[8];
+                    const float4 b0 = *reinterpret_cast<const float4*>(bias_s + co);
+                    const float4 b1 = *reinterpret_cast<const float4*>(bias_s + co + 4);
+                    a[0] = v[g * 8 + 0] + b0.x; a[1] = v[g * 8 + 1] + b0.y; a[2] = v[g * 8 + 2] + b0.z; a[3] = v[g * 8 + 3] + b0.w;
+                    a[4] = v[g * 8 + 4] + b1.x; a[5] = v[g * 8 + 5] + b1.y; a[6] = v[g * 8 + 6] + b1.z; a[7] = v[g * 8 + 7] + b1.w;
+                    if (RES) {
+                        if (valid && co < p.Cout) {
+                            const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.res + pix * p.Cout + co));
+                            const __half2* rh = reinterpret_cast<const __half2*>(&rv);
 #pragma unroll
-                        for (int e = 0; e < 4; e++) {
-                            const float2 f = __half22float2(rh[e]);
-                            vv[2 * e] += f.x;
-                            vv[2 * e + 1] += f.y;
+                            for (int e = 0; e < 4; e++) {
+                                const float2 f = __half22float2(rh[e]);
+                                a[2 * e] += f.x;
+                                a[2 * e + 1] += f.y;
+                            }
                         }
                     }
                     uint4 o;
                     uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
                     for (int e = 0; e < 4; e++) {
-                        float a0 = apply_act(vv[2 * e], p.act), a1 = apply_act(vv[2 * e + 1], p.act);
-                        if (p.pool) {
-                            // round first, then take the max over the 2x2 window held by this warp
-                            __half2 hv = __floats2half2_rn(a0, a1);
-                            __half2 o1 = __shfl_xor_sync(0xffffffffu, hv, 1);
-                            hv = __hmax2(hv, o1);
-                            o1 = __shfl_xor_sync(0xffffffffu, hv, p.TW);
-                            hv = __hmax2(hv, o1);
-                            ou[e] = *reinterpret_cast<uint32_t*>(&hv);
-                        } else {
-                            ou[e] = pack_half2(a0, a1);
+                        __half2 hv = __floats2half2_rn(act_t<ACT>(a[2 * e]), act_t<ACT>(a[2 * e + 1]));
+                        if (POOL) {  // rounded first, then the max over the 2x2 window held by this warp
+                            hv = __hmax2(hv, __shfl_xor_sync(0xffffffffu, hv, 1));
+                            hv = __hmax2(hv, __shfl_xor_sync(0xffffffffu, hv, p.TW));
                         }
+                        ou[e] = *reinterpret_cast<uint32_t*>(&hv);
                     }
-                    if (writer) *reinterpret_cast<uint4*>(p.out + opix * p.Cout + co + h8 * 8) = o;
+                    if (POOL) {
+                        if (writer && co < p.Cout) *reinterpret_cast<uint4*>(p.out + opix * p.Cout + co) = o;
+                    } else {
+                        const int g8 = (cc >> 3) + g;
+                        *reinterpret_cast<uint4*>(stage_out + (g8 >> 3) * kABytes + m * 128 + (((g8 & 7) ^ (m & 7)) << 4)) = o;
+                    }
                 }
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tempty_bar[acc]);
-            if (j == 0 && threadIdx.x == 64) DLF_TRACE_POINT(p.status, 6);
+            if (lane == 0) mbar_arrive(&tempty_bar[acc]);  // the accumulator is drained
+            if (!POOL) {
+                fence_proxy_async_smem();  // the staging tile is read by the TMA unit
+                epi_bar_sync();
+                if (issuer) {
+                    for (int pl = 0; pl * 64 < ncols; pl++)
+                        tma_store_4d(&tmy, stage_out + pl * kABytes, c.co0 + pl * 64, c.wo0, c.ho0, c.n0);
+                    tma_store_commit();
+                    tma_store_wait_read();
+                }
+                epi_bar_sync();  // the staging tile may be overwritten
+            }
+            if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 6);
         }
+        if (!POOL && issuer) tma_store_wait_all();
     }
 
     tc_fence_before_sync();
@@ -257,11 +292,27 @@ Tile pick_tile(int N, int Ho, int Wo, int pool) {
     return best;
 }
 
+typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const ConvTcParams);
+
+template <int ACT, bool POOL>
+KernelFn pick_res(bool res) {
+    return res ? conv_tc_kernel<ACT, POOL, true> : conv_tc_kernel<ACT, POOL, false>;
+}
+template <int ACT>
+KernelFn pick_pool(bool pool, bool res) {
+    return pool ? pick_res<ACT, true>(res) : pick_res<ACT, false>(res);
+}
+KernelFn pick_kernel(int act, bool pool, bool res) {
+    if (act == 0) return pick_pool<0>(pool, res);
+    if (act == 1) return pick_pool<1>(pool, res);
+    return pick_pool<2>(pool, res);
+}
+
 }  // namespace
 
 bool conv_tc_supported(const ConvArgs& a) {
     if (a.groups != 1) return false;
-    if (a.Cin % 8 || a.Cout % 8) return false;
+    if (a.Cin % 8 || a.Cout % 8 || a.Cout > 4096) return false;
     if (a.stride < 1 || a.stride > 2) return false;
     if (a.kh * a.kw > 49) return false;
     if (a.N < 1 || a.Ho < 1 || a.Wo < 1) return false;
@@ -284,13 +335,20 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     p.tiles_n = (a.N + tl.tn - 1) / tl.tn;
     const int cout16 = (a.Cout + 15) / 16 * 16;
     p.n_tiles_n = (cout16 + 255) / 256;
-    p.BN = ((cout16 + p.n_tiles_n - 1) / p.n_tiles_n + 15) / 16 * 16;
+    // several channel tiles: a multiple of 64 each, so that a tile's 64-channel TMA store boxes never
+    // reach into its neighbour's channels
+    p.BN = p.n_tiles_n == 1 ? cout16 : std::min(256, ((cout16 + p.n_tiles_n - 1) / p.n_tiles_n + 63) / 64 * 64);
+    p.n_tiles_n = (cout16 + p.BN - 1) / p.BN;
     p.kchunks = (a.Cin + 63) / 64;
     p.ksteps_last = ((a.Cin - (p.kchunks - 1) * 64) + 15) / 16;
-    p.act = a.act; p.pool = a.pool;
     const int stage_bytes = kABytes + p.BN * 128;
-    p.stages = std::min(6, (kMaxSmem - 1024) / stage_bytes);
+    const int out_planes = a.pool ? 0 : (p.BN + 63) / 64;
+    const int bias_bytes = (p.n_tiles_n * p.BN * 4 + 1023) / 1024 * 1024;
+    const int fixed = out_planes * kABytes + bias_bytes + 1024;
+    p.stages = std::min(6, (kMaxSmem - fixed) / stage_bytes);
     p.stages = std::max(1, std::min(p.stages, a.kh * a.kw * p.kchunks));
+    p.stage_out_off = p.stages * stage_bytes;
+    p.bias_off = p.stage_out_off + out_planes * kABytes;
     const long long n_work = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n * p.n_tiles_n;
     if (n_work > 0x7fffffffLL) return DLF_E_UNSUPPORTED;
     p.n_work = static_cast<int>(n_work);
@@ -301,7 +359,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     p.bias = a.bias; p.res = static_cast<const __half*>(a.res); p.out = static_cast<__half*>(a.y);
     p.status = status_dev;
 
-    CUtensorMap tmx, tmw;
+    CUtensorMap tmx, tmw, tmy;
     {
         const uint64_t dims[4] = {static_cast<uint64_t>(a.Cin), static_cast<uint64_t>(a.W), static_cast<uint64_t>(a.H),
                                   static_cast<uint64_t>(a.N)};
@@ -322,9 +380,20 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         int rc = encode_tmap(&tmw, a.w, 3, dims, strides, box, es);
         if (rc) return rc;
     }
+    {   // output map (unused by the pooled variant, which stores from registers)
+        const int Hy = a.pool ? a.Ho / 2 : a.Ho, Wy = a.pool ? a.Wo / 2 : a.Wo;
+        const uint64_t dims[4] = {static_cast<uint64_t>(a.Cout), static_cast<uint64_t>(Wy), static_cast<uint64_t>(Hy),
+                                  static_cast<uint64_t>(a.N)};
+        const uint64_t strides[3] = {static_cast<uint64_t>(a.Cout) * 2, static_cast<uint64_t>(Wy) * a.Cout * 2,
+                                     static_cast<uint64_t>(Hy) * Wy * a.Cout * 2};
+        const uint32_t box[4] = {64, static_cast<uint32_t>(tl.tw), static_cast<uint32_t>(tl.th), static_cast<uint32_t>(tl.tn)};
+        const uint32_t es[4] = {1, 1, 1, 1};
+        int rc = encode_tmap(&tmy, a.y, 4, dims, strides, box, es);
+        if (rc) return rc;
+    }
     const int grid = std::max(1, std::min(sm_count, p.n_work));
-    const size_t smem = std::max<size_t>(static_cast<size_t>(p.stages) * stage_bytes + 1024, 120 * 1024);
-    conv_tc_kernel<<<grid, kThreads, smem, s>>>(tmx, tmw, p);
+    const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024, 120 * 1024);
+    pick_kernel(a.act, a.pool != 0, a.res != nullptr)<<<grid, kThreads, smem, s>>>(tmx, tmw, tmy, p);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
@@ -332,8 +401,13 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
 int conv_tc_init() {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-        if (e != cudaSuccess) return cuda_fail(e);
+        for (int act = 0; act < 3; act++)
+            for (int pool = 0; pool < 2; pool++)
+                for (int res = 0; res < 2; res++) {
+                    cudaError_t e = cudaFuncSetAttribute(pick_kernel(act, pool != 0, res != 0),
+                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+                    if (e != cudaSuccess) return cuda_fail(e);
+                }
         attr_set = true;
     }
     return DLF_OK;
