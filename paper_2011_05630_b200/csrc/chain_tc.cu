@@ -21,9 +21,10 @@
 // global memory.  Weights stream through a TMA ring, once per pass; the next tile's input frame
 // is prefetched into a second buffer while the current tile computes.
 //
-// Warp roles: 0 weight producer, 1 UMMA issuer (owns the TMEM allocation), 2-9 epilogue (two per
-// TMEM lane quarter, alternating 32-column chunks), 10 input producer.  The epilogue is
-// specialised at compile time on (activation, destination): see epi_pass.
+// Warp roles: 0-7 epilogue (two per TMEM lane quarter, alternating 32-column chunks), 8 UMMA
+// issuer, 9-10 weight producers, 11 input producer.  Measured on B200: one TMA instruction
+// keeps its issuing thread busy for about 0.28 us whatever the box size, so weights travel in
+// boxes of several taps / K chunks (up to 32 KB) and the loads are spread over several warps.
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -38,9 +39,12 @@ namespace dlf {
 
 namespace {
 
-constexpr int kEpiWarps = 8;
-constexpr int kThreads = 64 + 32 * kEpiWarps + 32;
-constexpr int kInputWarp = 2 + kEpiWarps;
+constexpr int kEpiWarps = 8;                 // warps 0..7: epilogue (warp & 3 = TMEM lane quarter)
+constexpr int kMmaWarp = kEpiWarps;          // warp 8: UMMA issuer, owns the TMEM allocation
+constexpr int kWeightWarp0 = kEpiWarps + 1;  // warps 9, 10: weight producers (alternate ring stages)
+constexpr int kInputWarp0 = kEpiWarps + 3;   // warp 11: input producer (one box per 64-channel plane, a tile ahead)
+constexpr int kThreads = 32 * (kEpiWarps + 4);
+constexpr int kWeightOpBytes = 32 * 1024;    // target size of one weight TMA box
 constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
 constexpr int kMaxBias = 4096;           // floats of bias staged in shared memory (all layers)
 
@@ -51,6 +55,7 @@ struct ChainLayerP {
     int n_pad;                 // cout rounded up to 16
     int n_chunks, chunk_n;     // channel chunks of chunk_n (the last one may be smaller)
     int slot, per_pass;        // TMEM columns per block, blocks per pass (half of TMEM)
+    int tg, kg, w_rank4;       // taps and K chunks per weight box; 4-d weight view (cin % 64 == 0)
     int bias_off;
     const float* bias;
 };
@@ -188,7 +193,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         fence_barrier_init();
         tma_prefetch_desc(&p.tmx);
     }
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
         tmem_alloc(&tmem_base_s, 512);
         tmem_relinquish();
     }
@@ -202,7 +207,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     const uint32_t tmem_base = tmem_base_s;
     const int frame_rows = p.rows * p.pitch;
 
-    if (warp == kInputWarp) {
+    if (warp >= kInputWarp0) {
         // ---- input producer: one frame per tile, prefetched into the free input buffer ---------
         if (lane == 0) {
             uint32_t tile_i = 0;
@@ -216,33 +221,36 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                                 &in_full_bar[ib], pl * 64, txi * p.tw - p.halo, tyi * p.th - p.halo, n);
             }
         }
-    } else if (warp == 0) {
-        // ---- weight producer: one [chunk_n][64] slab per (tap, K chunk) of every pass ---------------
+    } else if (warp >= kWeightWarp0) {
+        // ---- weight producers: one box of tg taps x kg K chunks x [chunk_n][64] per ring stage ------
         if (lane == 0) {
+            const uint32_t parity = warp - kWeightWarp0;
             uint32_t wit = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
                 for (int l = 0; l < p.n_layers && ok; l++) {
                     const ChainLayerP& L = p.L[l];
                     const int passes = (L.nb + L.per_pass - 1) / L.per_pass;
-                    for (int c = 0; c < L.n_chunks && ok; c++) {
-                        const uint32_t bytes = static_cast<uint32_t>(L.chunk_n) * 128u;  // the whole box, rows past cout zero-filled
+                    const uint32_t bytes = static_cast<uint32_t>(L.tg * L.kg * L.chunk_n) * 128u;  // the whole box
+                    for (int c = 0; c < L.n_chunks && ok; c++)
                         for (int ps = 0; ps < passes && ok; ps++)
-                            for (int tap = 0; tap < L.k * L.k && ok; tap++)
-                                for (int kc = 0; kc < L.kchunks; kc++, wit++) {
+                            for (int t0 = 0; t0 < L.k * L.k && ok; t0 += L.tg)
+                                for (int g0 = 0; g0 < L.kchunks; g0 += L.kg, wit++) {
                                     const int st = wit % p.stages;
+                                    // a ring stage belongs to one producer (see the parity of mbarrier waits)
+                                    if ((st & 1u) != parity) continue;
                                     ok = mbar_wait(&wempty_bar[st], ((wit / p.stages) & 1u) ^ 1u, abort_flag, p.status,
                                                    0x200 | (blockIdx.x << 12));
                                     if (!ok) break;
                                     mbar_expect_tx(&wfull_bar[st], bytes);
-                                    tma_load_3d(sbase + p.ring_off + static_cast<size_t>(st) * p.stage_bytes, &p.tmw[l],
-                                                &wfull_bar[st], kc * 64, tap, c * L.chunk_n);
+                                    uint8_t* dst = sbase + p.ring_off + static_cast<size_t>(st) * p.stage_bytes;
+                                    if (L.w_rank4) tma_load_4d(dst, &p.tmw[l], &wfull_bar[st], 0, c * L.chunk_n, t0, g0);
+                                    else tma_load_3d(dst, &p.tmw[l], &wfull_bar[st], g0 * 64, c * L.chunk_n, t0);
                                 }
-                    }
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == kMmaWarp) {
         // ---- UMMA issuer ------------------------------------------------------------------------------------
         if (lane == 0) {
             uint32_t wit = 0, tile_i = 0, pass_i = 0, act_i = 0;
@@ -268,28 +276,35 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                                            0x500 | (blockIdx.x << 12));
                             if (!ok) break;
                             tc_fence_after_sync();
-                            for (int tap = 0; tap < L.k * L.k && ok; tap++) {
-                                const int r = tap / L.k, s = tap % L.k;
-                                const int shift = (r - L.pad) * p.pitch + (s - L.pad);
-                                for (int kc = 0; kc < L.kchunks; kc++, wit++) {
+                            for (int t0 = 0; t0 < L.k * L.k && ok; t0 += L.tg) {
+                                for (int g0 = 0; g0 < L.kchunks; g0 += L.kg, wit++) {
                                     const int st = wit % p.stages;
                                     ok = mbar_wait(&wfull_bar[st], (wit / p.stages) & 1u, abort_flag, p.status,
                                                    0x600 | (blockIdx.x << 12));
                                     if (!ok) break;
                                     tc_fence_after_sync();
-                                    const uint32_t b_lo = umma_desc_lo(base + p.ring_off + st * p.stage_bytes);
-                                    const int ksteps = (kc == L.kchunks - 1) ? L.ksteps_last : 4;
-                                    const uint32_t arow0 = abuf + kc * p.plane_bytes + (L.qs + b0 * 128 + shift) * 128;
-                                    const uint32_t acc0 = (tap | kc) != 0;
-                                    uint32_t d_tmem = tmem_base + half * 256u;
-                                    for (int b = 0; b < nblk; b++, d_tmem += L.slot) {
-                                        const uint32_t arow = arow0 + b * (128 * 128);
-                                        const uint32_t a_lo = umma_desc_lo(arow);
-                                        const uint32_t a_hi = p.base_offset_mode ? (kDescHiSw128 | (((arow >> 7) & 7u) << 17)) : kDescHiSw128;
-                                        umma_f16_lo(d_tmem, a_lo, a_hi, b_lo, idesc, acc0);
-                                        if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, a_hi, b_lo + 2, idesc, 1);
-                                        if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, a_hi, b_lo + 4, idesc, 1);
-                                        if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, a_hi, b_lo + 6, idesc, 1);
+                                    const uint32_t wsm = base + p.ring_off + st * p.stage_bytes;
+                                    for (int g = 0; g < L.kg && g0 + g < L.kchunks; g++) {
+                                        const int kc = g0 + g;
+                                        const int ksteps = (kc == L.kchunks - 1) ? L.ksteps_last : 4;
+                                        for (int tt = 0; tt < L.tg; tt++) {
+                                            const int tap = t0 + tt;
+                                            const int r = tap / L.k, sx = tap - r * L.k;
+                                            const int shift = (r - L.pad) * p.pitch + (sx - L.pad);
+                                            const uint32_t b_lo = umma_desc_lo(wsm + (g * L.tg + tt) * L.chunk_n * 128);
+                                            const uint32_t arow0 = abuf + kc * p.plane_bytes + (L.qs + b0 * 128 + shift) * 128;
+                                            const uint32_t acc0 = (tap | kc) != 0;
+                                            uint32_t d_tmem = tmem_base + half * 256u;
+                                            for (int b = 0; b < nblk; b++, d_tmem += L.slot) {
+                                                const uint32_t arow = arow0 + b * (128 * 128);
+                                                const uint32_t a_lo = umma_desc_lo(arow);
+                                                const uint32_t a_hi = p.base_offset_mode ? (kDescHiSw128 | (((arow >> 7) & 7u) << 17)) : kDescHiSw128;
+                                                umma_f16_lo(d_tmem, a_lo, a_hi, b_lo, idesc, acc0);
+                                                if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, a_hi, b_lo + 2, idesc, 1);
+                                                if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, a_hi, b_lo + 4, idesc, 1);
+                                                if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, a_hi, b_lo + 6, idesc, 1);
+                                            }
+                                        }
                                     }
                                     umma_commit(&wempty_bar[st]);
                                 }
@@ -304,10 +319,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         }
     } else {
         // ---- epilogue warps ------------------------------------------------------------------------------------
-        const int et = threadIdx.x - 64;  // 0 .. 32*kEpiWarps-1
+        const int et = threadIdx.x;  // 0 .. 32*kEpiWarps-1
         EpiCtx cx;
         cx.row = (warp & 3) * 32 + lane;
-        cx.half = (warp - 2) >> 2;
+        cx.half = warp >> 2;
         cx.tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         uint32_t pass_i = 0;
         bool ok = true;
@@ -385,7 +400,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
         if (abort_s) __nanosleep(20000);  // let copies in flight land before the CTA retires
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, 512);
@@ -398,6 +413,26 @@ int pad16(int c) { return (c + 15) / 16 * 16; }
 struct LayerGeom {
     int qs, range, nb, n_pad, n_chunks, chunk_n, slot, per_pass;
 };
+
+struct WeightBox {
+    int tg, kg, rank4, bytes;
+};
+
+// Taps and K chunks per weight TMA box: as many as fit the target size, whole kernel rows first.
+WeightBox weight_box(int cin, int cout, int k) {
+    WeightBox w;
+    const int n_pad = pad16(cout), chunk = n_pad > 256 ? 256 : n_pad;
+    const int kchunks = planes_of(cin);
+    w.rank4 = (cin % 64 == 0) ? 1 : 0;
+    w.tg = 1;
+    for (int t : {k * k, k}) {
+        if (t * chunk * 128 <= kWeightOpBytes) { w.tg = t; break; }
+    }
+    w.kg = 1;
+    if (w.rank4 && (w.tg == k * k || k == 1)) w.kg = std::max(1, std::min(kchunks, kWeightOpBytes / (w.tg * chunk * 128)));
+    w.bytes = w.tg * w.kg * chunk * 128;
+    return w;
+}
 
 LayerGeom layer_geom(int cout, int cum_pad, int rows, int pitch) {
     LayerGeom g;
@@ -459,7 +494,7 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
         if (l > 0 && a.cin[l] != a.cout[l - 1]) return best;
         halo += a.k[l] / 2;
         bias_floats += pad16(a.cout[l]);
-        stage_n = std::max(stage_n, std::min(pad16(a.cout[l]), 256));
+        stage_n = std::max(stage_n, weight_box(a.cin[l], a.cout[l], a.k[l]).bytes / 128);
     }
     if (bias_floats > kMaxBias) return best;
     const int L = a.n_layers;
@@ -482,7 +517,7 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
             if (n_tiles > 0x7fffffffLL) continue;
             const long long waves = (n_tiles + sm_count - 1) / sm_count;
             for (int in_bufs = 2; in_bufs >= 1; in_bufs--) {
-                int stages = 6;
+                int stages = 3;
                 auto total = [&](int st) { return fixed + static_cast<size_t>(in_bufs) * in_planes * plane + static_cast<size_t>(st) * stage_bytes; };
                 while (stages > 2 && total(stages) > static_cast<size_t>(kMaxSmem)) stages--;
                 if (total(stages) > static_cast<size_t>(kMaxSmem)) continue;
@@ -558,12 +593,24 @@ int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int 
         L.bias_off = boff;
         boff += g.n_pad;
         L.bias = a.bias[l];
+        const WeightBox wb = weight_box(a.cin[l], a.cout[l], a.k[l]);
+        L.tg = wb.tg; L.kg = wb.kg; L.w_rank4 = wb.rank4;
         const uint64_t taps = static_cast<uint64_t>(a.k[l]) * a.k[l];
-        const uint64_t dims[3] = {static_cast<uint64_t>(a.cin[l]), taps, static_cast<uint64_t>(a.cout[l])};
-        const uint64_t strides[2] = {static_cast<uint64_t>(a.cin[l]) * 2, taps * a.cin[l] * 2};
-        const uint32_t box[3] = {64, 1, static_cast<uint32_t>(std::min(g.chunk_n, g.n_pad))};
-        const uint32_t es[3] = {1, 1, 1};
-        int rc = encode_tmap(&p.tmw[l], a.w[l], 3, dims, strides, box, es);
+        const uint32_t box_n = static_cast<uint32_t>(std::min(g.chunk_n, g.n_pad));
+        int rc;
+        if (wb.rank4) {  // [cout][tap][cin] seen as (64 channels, cout, tap, cin / 64)
+            const uint64_t dims[4] = {64, static_cast<uint64_t>(a.cout[l]), taps, static_cast<uint64_t>(a.cin[l] / 64)};
+            const uint64_t strides[3] = {taps * a.cin[l] * 2, static_cast<uint64_t>(a.cin[l]) * 2, 128};
+            const uint32_t box[4] = {64, box_n, static_cast<uint32_t>(wb.tg), static_cast<uint32_t>(wb.kg)};
+            const uint32_t es[4] = {1, 1, 1, 1};
+            rc = encode_tmap(&p.tmw[l], a.w[l], 4, dims, strides, box, es);
+        } else {         // (cin, cout, tap): K chunks are addressed along dimension 0, zero-filled past cin
+            const uint64_t dims[3] = {static_cast<uint64_t>(a.cin[l]), static_cast<uint64_t>(a.cout[l]), taps};
+            const uint64_t strides[2] = {taps * a.cin[l] * 2, static_cast<uint64_t>(a.cin[l]) * 2};
+            const uint32_t box[3] = {64, box_n, static_cast<uint32_t>(wb.tg)};
+            const uint32_t es[3] = {1, 1, 1};
+            rc = encode_tmap(&p.tmw[l], a.w[l], 3, dims, strides, box, es);
+        }
         if (rc) return rc;
     }
     p.bias_floats = boff;

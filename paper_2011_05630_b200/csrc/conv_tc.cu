@@ -5,7 +5,9 @@
 //   M = 128 output pixels (a TN x TH x TW patch), N = up to 256 output channels, K = taps x C_in.
 //
 // A persistent grid of `sm_count` CTAs (the SM-count knob) walks the (pixel tile, channel tile)
-// work list.  Per CTA: one producer thread issues TMA tiled loads (the tap's shifted, strided
+// work list.  Per CTA: four producer threads (measured on B200: one TMA instruction keeps its
+// issuing thread busy for about 0.28 us whatever the box size, so the loads of a stage are spread
+// over several warps) issue TMA tiled loads (the tap's shifted, strided
 // window of the NHWC input, zero-filled outside the image = the convolution's padding; and the
 // tap's [C_out][64] weight slab) into a ring of 128-byte-swizzled stages; one thread issues
 // tcgen05.mma (fp16 x fp16 -> fp32) into one of two TMEM accumulators; eight epilogue warps (two
@@ -28,7 +30,9 @@ namespace dlf {
 namespace {
 
 constexpr int kEpiWarps = 8;
-constexpr int kThreads = 64 + 32 * kEpiWarps;
+constexpr int kMmaWarp = kEpiWarps;         // warps 0..7 epilogue (warp & 3 = TMEM lane quarter), 8 UMMA issuer,
+constexpr int kProdWarp0 = kEpiWarps + 1;   // 9..12 producers: A even / A odd / B even / B odd ring stages
+constexpr int kThreads = 32 * (kEpiWarps + 5);
 constexpr int kABytes = 128 * 128;  // 128 pixels x 64 fp16
 constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
 
@@ -86,7 +90,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     if (threadIdx.x == 0) {
         abort_s = 0;
         for (int i = 0; i < p.stages; i++) {
-            mbar_init(&full_bar[i], 1);
+            mbar_init(&full_bar[i], 2);  // the A and the B producer each arrive with their byte count
             mbar_init(&empty_bar[i], 1);
         }
         for (int i = 0; i < 2; i++) {
@@ -98,7 +102,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         tma_prefetch_desc(&tmw);
         if (!POOL) tma_prefetch_desc(&tmy);
     }
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
         tmem_alloc(&tmem_base_s, p.tmem_cols);
         tmem_relinquish();
     }
@@ -114,9 +118,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     const int taps = p.kh * p.kw;
     const int k_iters = taps * p.kchunks;
 
-    if (warp == 0) {
-        // ---- producer: TMA loads into the stage ring ------------------------------------------
+    if (warp >= kProdWarp0) {
+        // ---- producers: TMA loads into the stage ring -------------------------------------------
         if (lane == 0) {
+            const int role = warp - kProdWarp0;
+            const bool is_b = role >= 2;
+            const uint32_t parity = role & 1;
+            const uint32_t my_bytes = is_b ? static_cast<uint32_t>(p.BN) * 128u : static_cast<uint32_t>(kABytes);
             uint32_t it = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x) {
@@ -125,20 +133,23 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     const int r = tap / p.kw, s = tap % p.kw;
                     for (int kc = 0; kc < p.kchunks; kc++, it++) {
                         const int st = it % p.stages;
+                        // a ring stage belongs to ONE producer of each kind: a thread that skipped a phase of
+                        // a stage's barrier could not tell "two phases ago" from "now" by parity
+                        if ((st & 1u) != parity) continue;
                         ok = mbar_wait(&empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status,
                                        0x100 | (blockIdx.x << 12));
                         if (!ok) break;
                         uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
-                        mbar_expect_tx(&full_bar[st], static_cast<uint32_t>(stage_bytes));
-                        tma_load_4d(sa, &tmx, &full_bar[st], kc * 64, c.wo0 * p.stride - p.pad + s,
-                                    c.ho0 * p.stride - p.pad + r, c.n0);
-                        tma_load_3d(sa + kABytes, &tmw, &full_bar[st], kc * 64, tap, c.co0);
+                        mbar_expect_tx(&full_bar[st], my_bytes);
+                        if (is_b) tma_load_3d(sa + kABytes, &tmw, &full_bar[st], kc * 64, tap, c.co0);
+                        else tma_load_4d(sa, &tmx, &full_bar[st], kc * 64, c.wo0 * p.stride - p.pad + s,
+                                         c.ho0 * p.stride - p.pad + r, c.n0);
                         if (it == 0) DLF_TRACE_POINT(p.status, 2);
                     }
                 }
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == kMmaWarp) {
         // ---- MMA issuer ---------------------------------------------------------------------------
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f16(p.BN);
@@ -173,12 +184,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     } else {
         // ---- epilogue warps ---------------------------------------------------------------------------
         const int q = warp & 3;              // TMEM lane quarter this warp may read
-        const int half = (warp - 2) >> 2;    // which of the alternating 32-column chunks
+        const int half = warp >> 2;          // which of the alternating 32-column chunks
         const int m = q * 32 + lane;
         const int tw = m % p.TW, th = (m / p.TW) % p.TH, tn = m / (p.TW * p.TH);
         const int Hp = POOL ? p.Ho / 2 : p.Ho, Wp = POOL ? p.Wo / 2 : p.Wo;
         uint8_t* stage_out = stage0 + p.stage_out_off;
-        const bool issuer = (threadIdx.x == 64);
+        const bool issuer = (threadIdx.x == 0);
         uint32_t j = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
@@ -247,9 +258,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             if (!POOL) {
                 fence_proxy_async_smem();  // the staging tile is read by the TMA unit
                 epi_bar_sync();
-                if (issuer) {
-                    for (int pl = 0; pl * 64 < ncols; pl++)
-                        tma_store_4d(&tmy, stage_out + pl * kABytes, c.co0 + pl * 64, c.wo0, c.ho0, c.n0);
+                if (lane == 0 && warp * 64 < ncols) {  // one 64-channel plane per warp: TMA issue is slow per thread
+                    tma_store_4d(&tmy, stage_out + warp * kABytes, c.co0 + warp * 64, c.wo0, c.ho0, c.n0);
                     tma_store_commit();
                     tma_store_wait_read();
                 }
@@ -257,12 +267,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             }
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 6);
         }
-        if (!POOL && issuer) tma_store_wait_all();
+        if (!POOL && lane == 0) tma_store_wait_all();
     }
 
     tc_fence_before_sync();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kMmaWarp) {
         if (abort_s) __nanosleep(20000);  // let copies in flight land before the CTA retires
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, p.tmem_cols);
