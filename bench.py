@@ -191,6 +191,7 @@ def main():
     ap.add_argument("--bruteforce", action="store_true", help="also time the reduced brute-force plan")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--groups", action="store_true", help="print the per-group table to stderr")
+    ap.add_argument("--op-critical", type=float, default=None, help="override Algorithm 1's critical operation count per SM")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     wl = args.workload
@@ -230,7 +231,7 @@ def main():
 
     results = {}
     plan_list = [("unfused", None, None)]
-    t_ends, t_sms = plans.tuned_plan(sess.net, len(layers))
+    t_ends, t_sms = plans.tuned_plan(sess.net, len(layers), **({} if args.op_critical is None else {"op_critical": args.op_critical}))
     plan_list.append(("tuned", t_ends, t_sms))
     if args.bruteforce:
         b_ends, b_sms, _ = B.net_bruteforce(sess.net, len(layers), plans.sm_fractions(sms), 4, xd.data_ptr(),
@@ -274,7 +275,19 @@ def main():
            "h2d_bytes_per_step": int(x.nbytes), "d2h_bytes_per_step": int(yh.numel() * 2)}
 
     if rank == 0:
+        def show(rows, title):
+            sys.stderr.write("---- %s plan ----\n" % title)
+            for r in rows:
+                sys.stderr.write("%-12s %3d-%3d sms=%3d %8.4f ms roof %8.4f ms frac %.3f %s red %.2f\n" % (
+                    r["k"], r["first"], r["last"], r["sms"], r["ms"], r["t_roof_ms"], r["t_roof_ms"] / max(r["ms"], 1e-9),
+                    r["bound"], r["redundancy"]))
+        if args.groups:
+            sess.set_plan(None, None)
+            show(group_report(sess, B, xd, flush, stream, pk), "unfused")
+            sess.set_plan(t_ends, t_sms)
         rows = group_report(sess, B, xd, flush, stream, pk)
+        if args.groups:
+            show(rows, "tuned")
         t_meas = sum(r["ms"] for r in rows)
         t_roof = sum(r["t_roof_ms"] for r in rows)
         by_kernel = {}
@@ -293,11 +306,6 @@ def main():
                     "frac": ach / peak, "traffic": None, "kernel": dom_name, "launches_per_step": dom["n"],
                     "share_of_step": dom["ms"] / t_meas, "peak_source": pk_kind + " (sustained)" if tensor_bound else pk_kind,
                     "network_frac": t_roof / t_meas}
-        if args.groups:
-            for r in rows:
-                sys.stderr.write("%-12s %3d-%3d sms=%3d %8.4f ms roof %8.4f ms frac %.3f %s red %.2f\n" % (
-                    r["k"], r["first"], r["last"], r["sms"], r["ms"], r["t_roof_ms"], r["t_roof_ms"] / max(r["ms"], 1e-9),
-                    r["bound"], r["redundancy"]))
         cpu = None
         if not args.no_cpu_baseline:
             v, n, cores = oracle_images_per_sec(layers, params, x)

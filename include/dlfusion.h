@@ -173,8 +173,8 @@ int dlf_net_boundary_tensor(const dlf_net* net, int layer, const void** dev_ptr,
 int dlf_net_group_model(const dlf_net* net, int group, int64_t* flops, int64_t* hbm_bytes,
                         double* redundancy, int* launches);
 
-/* Name of the kernel variant that runs group g ("chain_tc", "conv_tc", "conv_direct", "dw3x3",
- * "fc", "maxpool", "gavgpool"); the string is owned by the library. */
+/* Name of the kernel variant that runs group g ("chain_tc", "conv_tc", "stem_tc", "conv_direct",
+ * "dw3x3", "fc", "maxpool", "gavgpool"); the string is owned by the library. */
 const char* dlf_net_group_kernel(const dlf_net* net, int group);
 
 /* Options (debugging and ablation); setting one clears the plan, which must be set again.

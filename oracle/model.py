@@ -19,7 +19,9 @@ block per forced segment, monotone block count).
 Readings where the printed algorithm is ambiguous (each is stated where it is used):
 the running sum of MPs is kept apart from its mean; the mean is not formed while a block
 holds no convolution / FC layer; indices run 0..n-1; a block's end index is inclusive and
-the tail is always closed; a caller-supplied rule can force a block to close.
+the tail is always closed; a caller-supplied rule can force a block to close; a block whose
+average MP reaches the core count of the chip gets the whole chip (the paper's top step, 32, is
+its whole chip; on a chip whose core count is not a power of two the floor would leave cores idle).
 """
 from __future__ import annotations
 
@@ -140,6 +142,8 @@ def algorithm1(kinds, channels, ops, p, must_close_after=None):
             if sum_op / avg_mp >= p["op_critical"] or forced:
                 partition.append(i)
                 mp = 2 ** int(math.floor(math.log2(avg_mp)))
+                if avg_mp >= p["s_max"]:  # the top step is the whole chip (32 of 32 cores in the paper)
+                    mp = p["s_max"]
                 mp_of_block.append(int(min(max(mp, 1), p["s_max"])))
                 sum_op, sum_mp, block_size, start = 0.0, 0.0, 0, i + 1
         elif forced:  # a block of layers without weights (a pool on its own)

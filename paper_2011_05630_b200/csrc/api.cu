@@ -58,8 +58,8 @@ int encode_tmap(void* out_map, const void* base, int rank, const uint64_t* dims,
     return DLF_OK;
 }
 
-enum Kind { K_CHAIN_TC, K_CONV_TC, K_CONV_DIRECT, K_DW, K_FC, K_MAXPOOL, K_GAVG };
-static const char* kKindName[] = {"chain_tc", "conv_tc", "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool"};
+enum Kind { K_CHAIN_TC, K_CONV_TC, K_CONV_DIRECT, K_DW, K_FC, K_MAXPOOL, K_GAVG, K_STEM_TC };
+static const char* kKindName[] = {"chain_tc", "conv_tc", "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool", "stem_tc"};
 
 struct Layer {
     dlf_layer_desc d;
@@ -210,7 +210,9 @@ static bool single_kind(const dlf_net* net, int i, Kind* kind) {
     switch (l.d.op) {
         case DLF_CONV: {
             ConvArgs a = conv_args(net, i, nullptr, nullptr);
+            if (l.d.res_src == -2) a.res = nullptr; else a.res = &a;  // only whether there is one matters here
             if (!net->opt_no_tc && conv_tc_supported(a)) { *kind = K_CONV_TC; return true; }
+            if (!net->opt_no_tc && stem_tc_supported(a)) { *kind = K_STEM_TC; return true; }
             if (l.d.groups > 1 && (l.d.cout / l.d.groups) % 16 != 0) return false;
             *kind = K_CONV_DIRECT;
             return true;
@@ -238,13 +240,18 @@ static bool single_kind(const dlf_net* net, int i, Kind* kind) {
 static bool make_group(const dlf_net* net, int first, int last, int sms, Group* g) {
     g->first = first; g->last = last; g->sms = sms;
     g->tiling = ChainTiling{};
-    if (first == last && !(net->opt_single_chain && !net->opt_no_tc && span_is_chain(net, first, last))) {
-        return single_kind(net, first, &g->kind);
+    if (first == last) {
+        // A single stride-1 3x3 layer with few channels re-reads its input nine times through the
+        // per-tap kernel; the fused-chain kernel loads the tile once (measured faster up to 64 channels).
+        const dlf_layer_desc& d = net->layers[first].d;
+        const bool prefer_chain = net->opt_single_chain || (d.op == DLF_CONV && d.kh == 3 && d.cin <= 64 && d.cout <= 64);
+        if (!(prefer_chain && !net->opt_no_tc && span_is_chain(net, first, last))) return single_kind(net, first, &g->kind);
     }
     if (net->opt_no_tc || !span_is_chain(net, first, last)) return false;
     ChainArgs a = chain_args(net, first, last, nullptr, nullptr);
     g->tiling = chain_tc_tiling(a, sms, net->dev_sms);
     g->kind = K_CHAIN_TC;
+    if (!g->tiling.ok && first == last) return single_kind(net, first, &g->kind);
     return g->tiling.ok;
 }
 
@@ -259,6 +266,7 @@ static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* 
             return launch_chain_tc(a, g.tiling, g.sms, net->opt_base_offset, status, s);
         }
         case K_CONV_TC: return launch_conv_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
+        case K_STEM_TC: return launch_stem_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
         case K_CONV_DIRECT: return launch_conv_direct(conv_args(net, g.first, in_dev, y), g.sms, s);
         case K_DW: return launch_dw3x3(conv_args(net, g.first, in_dev, y), g.sms, s);
         case K_FC: {
@@ -284,7 +292,8 @@ static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* 
 namespace dlf {
 int kernels_init() {
     int rc = conv_tc_init();
-    return rc ? rc : chain_tc_init();
+    if (rc == DLF_OK) rc = chain_tc_init();
+    return rc ? rc : stem_tc_init();
 }
 
 static void invalidate_graphs(dlf_net* net) {
@@ -635,6 +644,7 @@ int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_
             if (sum_op / avg >= params->op_critical || forced) {
                 group_end[ng] = i;
                 int mp = 1 << static_cast<int>(std::floor(std::log2(avg)));
+                if (avg >= s_max) mp = s_max;  // the top step is the whole chip, as 32 of 32 cores in the paper
                 sm_count[ng] = std::min(std::max(mp, 1), s_max);
                 ng++;
                 sum_op = sum_mp = 0.0;

@@ -76,6 +76,11 @@ bool conv_tc_supported(const ConvArgs& a);
 bool chain_tc_layer_supported(int cin, int cout, int k);
 int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s);
 
+// stem_tc.cu
+bool stem_tc_supported(const ConvArgs& a);
+int stem_tc_init();
+int launch_stem_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s);
+
 // chain_tc.cu
 ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms);
 int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int base_offset_mode, int* status_dev,

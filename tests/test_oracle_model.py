@@ -148,7 +148,7 @@ def test_algorithm1_structure(layers):
     for crit in (1.0, 1e6, 1e8, 1e9, 1e10, 1e12, 1e30):
         part, mps = model.algorithm1(kinds, ch, ops, dict(P, op_critical=crit))
         assert part[-1] == n - 1 and part == sorted(set(part)) and len(mps) == len(part)
-        assert all(m >= 1 and m <= 32 and (m & (m - 1)) == 0 for m in mps)
+        assert all(1 <= m <= 32 and (m & (m - 1)) == 0 for m in mps)
         if last is not None:
             assert len(part) <= last
         last = len(part)
