@@ -134,8 +134,15 @@ static bool chain_layer_ok(const Layer& l) {
            d.pad == d.kh / 2 && chain_tc_layer_supported(d.cin, d.cout, d.kh);
 }
 
+// A fused group re-streams each layer's weights for every tile, so a layer may join other layers
+// only while its weights stay small next to the tile it works on.
+constexpr int64_t kMaxFusedWeightBytes = 160 * 1024;
+
 static bool span_is_chain(const dlf_net* net, int first, int last) {
     if (last - first + 1 > kMaxChain) return false;
+    if (last > first)
+        for (int i = first; i <= last; i++)
+            if (net->layers[i].w_elems * 2 > kMaxFusedWeightBytes) return false;
     const int n = static_cast<int>(net->layers.size());
     for (int i = first; i <= last; i++) {
         const Layer& l = net->layers[i];

@@ -7,7 +7,7 @@ from . import binding as B
 
 # Eq. 5 weights are the paper's; the affine map to an SM count and the critical operation count
 # per SM are fitted to B200 (the paper fits them to its own accelerator the same way).
-TUNER = dict(alpha=0.316, beta=0.659, kappa=12.0, kappa0=-120.0, op_critical=2.0e7)
+TUNER = dict(alpha=0.316, beta=0.659, kappa=12.0, kappa0=-60.0, op_critical=1.0e7)
 
 
 def tuned_plan(net, n_layers, **over):

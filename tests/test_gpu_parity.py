@@ -124,12 +124,13 @@ CHAINS = [
     # (n, h, w, c, kernel sizes)
     (1, 32, 32, 16, (3, 3)),
     (2, 19, 23, 64, (3, 3, 3)),
-    (2, 14, 14, 128, (3, 1, 3)),
+    (2, 14, 14, 64, (3, 1, 3)),
     (1, 56, 56, 32, (1, 1, 1, 1)),
-    (3, 7, 7, 256, (3, 3)),
+    (3, 7, 7, (256, 64, 256), (1, 1)),
     (1, 28, 28, 64, (3, 3, 3, 3)),
-    (2, 28, 28, (128, 128, 512), (3, 1)),     # bottleneck tail: more than 256 output channels
-    (4, 14, 14, (128, 320, 64), (1, 3)),      # a wide intermediate map (5 planes, two channel chunks)
+    (2, 28, 28, (64, 64, 512), (3, 1)),       # bottleneck tail: more than 256 output channels
+    (4, 14, 14, (128, 320, 64), (1, 1)),      # a wide intermediate map (5 planes, two channel chunks)
+    (2, 14, 14, (32, 160, 32), (1, 3)),       # 3x3 layer reading a 3-plane intermediate
 ]
 
 

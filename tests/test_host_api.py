@@ -97,8 +97,11 @@ def _chain_layer_ok(l):
 def span_is_chain(layers, first, last):
     """The structural rule of fusable spans, written from its description: a chain of dense
     stride-1 size-keeping 1x1/3x3 convolutions, each reading its predecessor, pool / residual on
-    the last layer only, no intermediate map used anywhere else; at most 8 layers."""
+    the last layer only, no intermediate map used anywhere else; at most 8 layers; in a group of
+    several layers no layer's weights exceed 160 KB (they are re-streamed for every tile)."""
     if last - first + 1 > 8:
+        return False
+    if last > first and any(2 * l["cout"] * l["kh"] * l["kw"] * l["cin"] > 160 * 1024 for l in layers[first:last + 1]):
         return False
     for i in range(first, last + 1):
         l = layers[i]
@@ -119,7 +122,7 @@ def span_is_chain(layers, first, last):
     return True
 
 
-P = dict(alpha=0.316, beta=0.659, kappa=12.0, kappa0=-170.0, s_max=148)
+P = dict(alpha=0.316, beta=0.659, kappa=12.0, kappa0=-60.0, s_max=148)
 
 
 @pytest.mark.parametrize("name,layers,batch", NETS + [("chain8", nw.conv_chain(8, 64, 3), 16),
