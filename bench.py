@@ -50,6 +50,29 @@ def build_layers(spec):
     return getattr(networks, spec)()
 
 
+def recorded_traffic(kernel, workload):
+    """DRAM bytes per step of `kernel` from the committed ncu summary, or None when there is no
+    summary for this kernel / workload or the kernel's source changed since the capture."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "%s_%s_dram.md" % (kernel, workload))
+    if not os.path.exists(path):
+        return None
+    vals = {}
+    for line in open(path):
+        parts = line.strip().split(":", 1)
+        if len(parts) == 2 and parts[0].strip().replace("_", "").isalnum():
+            vals[parts[0].strip()] = parts[1].split("(")[0].strip()
+    try:
+        h = hashlib.sha256()
+        for f in ("%s.cu" % kernel, "ptx.cuh"):
+            h.update(open(os.path.join(ROOT, "paper_2011_05630_b200", "csrc", f), "rb").read())
+        if h.hexdigest()[:16] != vals["source_sha256_16"]:
+            return None
+        return float(vals["traffic_bytes_per_step"]) / float(vals["launches_per_step"])
+    except Exception:
+        return None
+
+
 def peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -303,7 +326,8 @@ def main():
         else:
             ach, peak, unit = dom["bytes"] / (dom["ms"] * 1e-3) / 1e9, pk["hbm_gbs"], "GB/s"
         roofline = {"bound": "tensor" if tensor_bound else "hbm", "achieved": ach, "peak": peak, "unit": unit,
-                    "frac": ach / peak, "traffic": None, "kernel": dom_name, "launches_per_step": dom["n"],
+                    "frac": ach / peak, "traffic": recorded_traffic(dom_name, wl), "traffic_unit": "bytes per launch (mean)",
+                    "kernel": dom_name, "launches_per_step": dom["n"],
                     "share_of_step": dom["ms"] / t_meas, "peak_source": pk_kind + " (sustained)" if tensor_bound else pk_kind,
                     "network_frac": t_roof / t_meas}
         cpu = None
