@@ -223,7 +223,7 @@ def main():
 
     import torch
     import torch.distributed as dist
-    from paper_2011_05630_b200 import binding as B, plans, synth
+    from paper_2011_05630_b200 import binding as B, dist as D, plans, synth
     from paper_2011_05630_b200.runtime import Session
 
     rank = int(os.environ.get("RANK", "0"))
@@ -271,11 +271,8 @@ def main():
         barrier()
         if name == "tuned":
             clocks = sampler.stop()
-        total = torch.tensor([sum(ms)], dtype=torch.float64, device=sess.device)
-        if world > 1:
-            dist.all_reduce(total, op=dist.ReduceOp.MAX)
-        results[name] = {"ms_per_step": float(total.item()) / args.steps, "n_groups": sess.n_groups,
-                         "value": world * batch * args.steps / (float(total.item()) * 1e-3)}
+        value, total_ms = D.job_throughput(sum(ms), batch * args.steps, device=sess.device)
+        results[name] = {"ms_per_step": total_ms / args.steps, "n_groups": sess.n_groups, "value": value}
 
     # end to end through the host-buffer entry point: pinned host input, H2D, run, D2H, per step
     sess.set_plan(t_ends, t_sms)
@@ -291,11 +288,8 @@ def main():
         B.net_run_host(sess.net, xh.data_ptr(), yh.data_ptr(), stream.cuda_stream)
     e1.record(stream)
     barrier()
-    e2e_ms = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=sess.device)
-    if world > 1:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e = {"value": world * batch * e2e_steps / (float(e2e_ms.item()) * 1e-3), "unit": "images/s",
-           "h2d_bytes_per_step": int(x.nbytes), "d2h_bytes_per_step": int(yh.numel() * 2)}
+    e2e_value, _ = D.job_throughput(e0.elapsed_time(e1), batch * e2e_steps, device=sess.device)
+    e2e = {"value": e2e_value, "unit": "images/s", "h2d_bytes_per_step": int(x.nbytes), "d2h_bytes_per_step": int(yh.numel() * 2)}
 
     if rank == 0:
         def show(rows, title):
