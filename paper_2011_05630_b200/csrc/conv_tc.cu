@@ -42,6 +42,7 @@ struct ConvTcParams {
     int TW, TH, TN, tiles_w, tiles_h, tiles_n;
     int BN, n_tiles_n, acc_stride;
     int kchunks, ksteps_last;
+    int kg, kgroups, grouped;  // K chunks per ring stage; stages per tap; 1 = 5-d / 4-d maps (cin % 64 == 0)
     int stages;
     int n_work;
     int stage_out_off, bias_off;  // byte offsets in dynamic shared memory
@@ -83,7 +84,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* stage0 = smem_raw + (base - smem_u32(smem_raw));
     float* bias_s = reinterpret_cast<float*>(stage0 + p.bias_off);
-    const int stage_bytes = kABytes + p.BN * 128;
+    const int stage_bytes = p.kg * (kABytes + p.BN * 128);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &abort_s;
 
@@ -116,7 +117,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
     const int taps = p.kh * p.kw;
-    const int k_iters = taps * p.kchunks;
+    const int k_iters = taps * p.kgroups;
 
     if (warp >= kProdWarp0) {
         // ---- producers: TMA loads into the stage ring -------------------------------------------
@@ -124,14 +125,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             const int role = warp - kProdWarp0;
             const bool is_b = role >= 2;
             const uint32_t parity = role & 1;
-            const uint32_t my_bytes = is_b ? static_cast<uint32_t>(p.BN) * 128u : static_cast<uint32_t>(kABytes);
+            const uint32_t my_bytes = static_cast<uint32_t>(p.kg) * (is_b ? static_cast<uint32_t>(p.BN) * 128u : static_cast<uint32_t>(kABytes));
             uint32_t it = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x) {
                 const TileCoord c = decode_work(p, t);
                 for (int tap = 0; tap < taps && ok; tap++) {
                     const int r = tap / p.kw, s = tap % p.kw;
-                    for (int kc = 0; kc < p.kchunks; kc++, it++) {
+                    for (int kq = 0; kq < p.kgroups; kq++, it++) {
                         const int st = it % p.stages;
                         // a ring stage belongs to ONE producer of each kind: a thread that skipped a phase of
                         // a stage's barrier could not tell "two phases ago" from "now" by parity
@@ -141,9 +142,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                         if (!ok) break;
                         uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
                         mbar_expect_tx(&full_bar[st], my_bytes);
-                        if (is_b) tma_load_3d(sa + kABytes, &tmw, &full_bar[st], kc * 64, tap, c.co0);
-                        else tma_load_4d(sa, &tmx, &full_bar[st], kc * 64, c.wo0 * p.stride - p.pad + s,
-                                         c.ho0 * p.stride - p.pad + r, c.n0);
+                        if (is_b) {
+                            if (p.grouped) tma_load_4d(sa + p.kg * kABytes, &tmw, &full_bar[st], 0, c.co0, tap, kq * p.kg);
+                            else tma_load_3d(sa + kABytes, &tmw, &full_bar[st], kq * 64, tap, c.co0);
+                        } else {
+                            const int wi = c.wo0 * p.stride - p.pad + s, hi = c.ho0 * p.stride - p.pad + r;
+                            if (p.grouped) tma_load_5d(sa, &tmx, &full_bar[st], 0, wi, hi, c.n0, kq * p.kg);
+                            else tma_load_4d(sa, &tmx, &full_bar[st], kq * 64, wi, hi, c.n0);
+                        }
                         if (it == 0) DLF_TRACE_POINT(p.status, 2);
                     }
                 }
@@ -161,21 +167,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + acc * p.acc_stride;
-                int kc = 0;
+                int kq = 0;
                 for (int ki = 0; ki < k_iters; ki++, it++) {
                     const int st = it % p.stages;
                     ok = mbar_wait(&full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                     if (!ok) break;
                     if (it == 0) DLF_TRACE_POINT(p.status, 3);
                     tc_fence_after_sync();
-                    const uint32_t a_lo = umma_desc_lo(base + st * stage_bytes), b_lo = umma_desc_lo(base + st * stage_bytes + kABytes);
-                    const int ksteps = (kc == p.kchunks - 1) ? p.ksteps_last : 4;
-                    umma_f16_lo(d_tmem, a_lo, kDescHiSw128, b_lo, idesc, ki != 0);
-                    if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, kDescHiSw128, b_lo + 2, idesc, 1);
-                    if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, kDescHiSw128, b_lo + 4, idesc, 1);
-                    if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, kDescHiSw128, b_lo + 6, idesc, 1);
+                    const uint32_t sa = base + st * stage_bytes, sb = sa + p.kg * kABytes;
+                    for (int g = 0; g < p.kg; g++) {
+                        const int kc = kq * p.kg + g;
+                        if (kc >= p.kchunks) break;
+                        const uint32_t a_lo = umma_desc_lo(sa + g * kABytes), b_lo = umma_desc_lo(sb + g * p.BN * 128);
+                        const int ksteps = (kc == p.kchunks - 1) ? p.ksteps_last : 4;
+                        umma_f16_lo(d_tmem, a_lo, kDescHiSw128, b_lo, idesc, (ki | g) != 0);
+                        if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, kDescHiSw128, b_lo + 2, idesc, 1);
+                        if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, kDescHiSw128, b_lo + 4, idesc, 1);
+                        if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, kDescHiSw128, b_lo + 6, idesc, 1);
+                    }
                     umma_commit(&empty_bar[st]);  // frees the stage once these MMAs have read it
-                    if (++kc == p.kchunks) kc = 0;
+                    if (++kq == p.kgroups) kq = 0;
                 }
                 if (ok) umma_commit(&tfull_bar[acc]);
                 if (j == 0) DLF_TRACE_POINT(p.status, 4);
@@ -344,19 +355,45 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     p.tiles_h = (a.Ho + tl.th - 1) / tl.th;
     p.tiles_n = (a.N + tl.tn - 1) / tl.tn;
     const int cout16 = (a.Cout + 15) / 16 * 16;
-    p.n_tiles_n = (cout16 + 255) / 256;
-    // several channel tiles: a multiple of 64 each, so that a tile's 64-channel TMA store boxes never
-    // reach into its neighbour's channels
-    p.BN = p.n_tiles_n == 1 ? cout16 : std::min(256, ((cout16 + p.n_tiles_n - 1) / p.n_tiles_n + 63) / 64 * 64);
-    p.n_tiles_n = (cout16 + p.BN - 1) / p.BN;
+    // Channel tile: layers with few pixel tiles (small images, small batch) get narrower channel tiles so
+    // that the work list covers the SMs; cost = waves x (tile width + a fixed per-item overhead).  With
+    // several channel tiles the width is a multiple of 64, so that a tile's 64-channel TMA store boxes
+    // never reach into its neighbour's channels.
+    {
+        const long long m_tiles = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n;
+        long long best_cost = -1;
+        for (int bn : {256, 192, 128, 64}) {
+            const int width = std::min(bn, cout16);
+            const int nt = (cout16 + width - 1) / width;
+            if (nt > 1 && width % 64) continue;
+            const long long waves = (m_tiles * nt + sm_count - 1) / sm_count;
+            const long long cost = waves * (width + 96);
+            if (best_cost < 0 || cost < best_cost) {
+                best_cost = cost;
+                p.BN = width;
+                p.n_tiles_n = nt;
+            }
+        }
+    }
     p.kchunks = (a.Cin + 63) / 64;
     p.ksteps_last = ((a.Cin - (p.kchunks - 1) * 64) + 15) / 16;
-    const int stage_bytes = kABytes + p.BN * 128;
     const int out_planes = a.pool ? 0 : (p.BN + 63) / 64;
     const int bias_bytes = (p.n_tiles_n * p.BN * 4 + 1023) / 1024 * 1024;
     const int fixed = out_planes * kABytes + bias_bytes + 1024;
+    // K chunks per ring stage: every stage costs the issuing threads a fixed handshake (barrier wait,
+    // TMA issue, commit), so a stage carries as many 64-channel chunks as leave room for >= 2 stages
+    p.grouped = (a.Cin % 64 == 0) ? 1 : 0;
+    p.kg = 1;
+    if (p.grouped)
+        for (int kg : {4, 2})
+            if (kg <= p.kchunks && 2 * kg * (kABytes + p.BN * 128) <= kMaxSmem - fixed && (kg == 2 || 3 * kg * (kABytes + p.BN * 128) <= kMaxSmem - fixed || a.kh * a.kw * ((p.kchunks + kg - 1) / kg) <= 2)) {
+                p.kg = kg;
+                break;
+            }
+    p.kgroups = (p.kchunks + p.kg - 1) / p.kg;
+    const int stage_bytes = p.kg * (kABytes + p.BN * 128);
     p.stages = std::min(6, (kMaxSmem - fixed) / stage_bytes);
-    p.stages = std::max(1, std::min(p.stages, a.kh * a.kw * p.kchunks));
+    p.stages = std::max(1, std::min(p.stages, a.kh * a.kw * p.kgroups));
     p.stage_out_off = p.stages * stage_bytes;
     p.bias_off = p.stage_out_off + out_planes * kABytes;
     const long long n_work = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n * p.n_tiles_n;
@@ -370,7 +407,26 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     p.status = status_dev;
 
     CUtensorMap tmx, tmw, tmy;
-    {
+    const uint64_t taps64 = static_cast<uint64_t>(a.kh) * a.kw;
+    if (p.grouped) {
+        // input seen as (64 channels, W, H, N, C_in / 64): one box carries kg chunks of a tap's window
+        const uint64_t dims[5] = {64, static_cast<uint64_t>(a.W), static_cast<uint64_t>(a.H), static_cast<uint64_t>(a.N),
+                                  static_cast<uint64_t>(a.Cin / 64)};
+        const uint64_t strides[4] = {static_cast<uint64_t>(a.Cin) * 2, static_cast<uint64_t>(a.W) * a.Cin * 2,
+                                     static_cast<uint64_t>(a.H) * a.W * a.Cin * 2, 128};
+        const uint32_t box[5] = {64, static_cast<uint32_t>(tl.tw * a.stride), static_cast<uint32_t>(tl.th * a.stride),
+                                 static_cast<uint32_t>(tl.tn), static_cast<uint32_t>(p.kg)};
+        const uint32_t es[5] = {1, static_cast<uint32_t>(a.stride), static_cast<uint32_t>(a.stride), 1, 1};
+        int rc = encode_tmap(&tmx, a.x, 5, dims, strides, box, es);
+        if (rc) return rc;
+        // weights [cout][tap][cin] seen as (64 channels, cout, tap, C_in / 64)
+        const uint64_t wdims[4] = {64, static_cast<uint64_t>(a.Cout), taps64, static_cast<uint64_t>(a.Cin / 64)};
+        const uint64_t wstrides[3] = {taps64 * a.Cin * 2, static_cast<uint64_t>(a.Cin) * 2, 128};
+        const uint32_t wbox[4] = {64, static_cast<uint32_t>(p.BN), 1, static_cast<uint32_t>(p.kg)};
+        const uint32_t wes[4] = {1, 1, 1, 1};
+        rc = encode_tmap(&tmw, a.w, 4, wdims, wstrides, wbox, wes);
+        if (rc) return rc;
+    } else {
         const uint64_t dims[4] = {static_cast<uint64_t>(a.Cin), static_cast<uint64_t>(a.W), static_cast<uint64_t>(a.H),
                                   static_cast<uint64_t>(a.N)};
         const uint64_t strides[3] = {static_cast<uint64_t>(a.Cin) * 2, static_cast<uint64_t>(a.W) * a.Cin * 2,
@@ -380,14 +436,11 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         const uint32_t es[4] = {1, static_cast<uint32_t>(a.stride), static_cast<uint32_t>(a.stride), 1};
         int rc = encode_tmap(&tmx, a.x, 4, dims, strides, box, es);
         if (rc) return rc;
-    }
-    {
-        const uint64_t taps = static_cast<uint64_t>(a.kh) * a.kw;
-        const uint64_t dims[3] = {static_cast<uint64_t>(a.Cin), taps, static_cast<uint64_t>(a.Cout)};
-        const uint64_t strides[2] = {static_cast<uint64_t>(a.Cin) * 2, taps * a.Cin * 2};
-        const uint32_t box[3] = {64, 1, static_cast<uint32_t>(p.BN)};
-        const uint32_t es[3] = {1, 1, 1};
-        int rc = encode_tmap(&tmw, a.w, 3, dims, strides, box, es);
+        const uint64_t wdims[3] = {static_cast<uint64_t>(a.Cin), taps64, static_cast<uint64_t>(a.Cout)};
+        const uint64_t wstrides[2] = {static_cast<uint64_t>(a.Cin) * 2, taps64 * a.Cin * 2};
+        const uint32_t wbox[3] = {64, 1, static_cast<uint32_t>(p.BN)};
+        const uint32_t wes[3] = {1, 1, 1};
+        rc = encode_tmap(&tmw, a.w, 3, wdims, wstrides, wbox, wes);
         if (rc) return rc;
     }
     {   // output map (unused by the pooled variant, which stores from registers)
