@@ -6,6 +6,8 @@
 // the work with a grid stride.
 #include <cuda_fp16.h>
 
+#include <algorithm>
+
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -106,53 +108,110 @@ __global__ void __launch_bounds__(128) conv_direct_kernel(ConvArgs a, long long 
 }
 
 // ---- depthwise 3x3 ------------------------------------------------------------------------------------
-// One thread = one output pixel x 8 channels: nine 128-bit loads, 72 fp32 multiply-adds.
-__global__ void __launch_bounds__(256) dw3x3_kernel(ConvArgs a, long long total) {
+// One thread = 8 channels x a strip of kDwStrip output columns of one output row.  The thread's 72
+// weights and 8 biases are converted to fp32 once (the launch makes the total thread count a
+// multiple of C/8, so a thread keeps its channels over the whole grid-stride loop); every input
+// vector of the strip's three rows is loaded once (128 bits), converted once and used by all the
+// outputs it touches.  Lanes run over the channel vectors first, so a warp reads contiguous NHWC
+// runs.  fp32 accumulation in (kh, kw) order, one rounding.
+constexpr int kDwStrip = 4;
+
+template <int STRIDE>
+__global__ void __launch_bounds__(128) dw3x3_kernel(ConvArgs a, long long total, int strips) {
+    constexpr int kCols = (kDwStrip - 1) * STRIDE + 3;  // input columns one strip reads per row
     const int c8n = a.Cout / 8;
-    for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < total;
-         i += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const int c8 = static_cast<int>(i % c8n);
-        long long p = i / c8n;
-        const int wo = static_cast<int>(p % a.Wo);
-        p /= a.Wo;
-        const int ho = static_cast<int>(p % a.Ho);
-        const int n = static_cast<int>(p / a.Ho);
-        const int c0 = c8 * 8;
-        // weights of channels c0..c0+7: 72 consecutive halves starting at c0*9
-        __align__(16) __half wv[72];
+    const long long tid = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x;
+    const long long nthreads = static_cast<long long>(gridDim.x) * blockDim.x;
+    if (tid >= total) return;
+    const int c0 = static_cast<int>(tid % c8n) * 8;
+    float w[9][8], b[8];
+    {
+        __align__(16) __half wv[72];  // weights of channels c0..c0+7: 72 consecutive halves starting at c0*9
         const uint4* wp4 = reinterpret_cast<const uint4*>(static_cast<const __half*>(a.w) + static_cast<long long>(c0) * 9);
 #pragma unroll
         for (int k = 0; k < 9; k++) reinterpret_cast<uint4*>(wv)[k] = __ldg(wp4 + k);
-        float acc[8];
 #pragma unroll
-        for (int j = 0; j < 8; j++) acc[j] = 0.0f;
+        for (int j = 0; j < 8; j++) {
+            b[j] = __ldg(a.bias + c0 + j);
+#pragma unroll
+            for (int t = 0; t < 9; t++) w[t][j] = __half2float(wv[j * 9 + t]);
+        }
+    }
+    const float lo = a.act >= 1 ? 0.0f : -INFINITY, hi = a.act == 2 ? 6.0f : INFINITY;
+    const __half* x = static_cast<const __half*>(a.x);
+    const __half* res = static_cast<const __half*>(a.res);
+    __half* y = static_cast<__half*>(a.y);
+    for (long long i = tid; i < total; i += nthreads) {
+        long long p = i / c8n;
+        const int strip = static_cast<int>(p % strips);
+        p /= strips;
+        const int ho = static_cast<int>(p % a.Ho);
+        const int n = static_cast<int>(p / a.Ho);
+        const int wo0 = strip * kDwStrip;
+        const int wi0 = wo0 * STRIDE - a.pad;
+        float acc[kDwStrip][8];
+#pragma unroll
+        for (int o = 0; o < kDwStrip; o++)
+#pragma unroll
+            for (int j = 0; j < 8; j++) acc[o][j] = 0.0f;
 #pragma unroll
         for (int r = 0; r < 3; r++) {
-            const int hi = ho * a.stride - a.pad + r;
-            if (hi < 0 || hi >= a.H) continue;
+            const int hi_ = ho * STRIDE - a.pad + r;
+            const bool row_ok = hi_ >= 0 && hi_ < a.H;
+            const __half* row = x + ((static_cast<long long>(n) * a.H + min(max(hi_, 0), a.H - 1)) * a.W) * a.Cin + c0;
+            // all loads of the row first, from clamped (always valid) addresses and without branches, so
+            // that they are in flight together; columns outside the image are zeroed afterwards
+            uint4 xv[kCols];
 #pragma unroll
-            for (int s = 0; s < 3; s++) {
-                const int wi = wo * a.stride - a.pad + s;
-                if (wi < 0 || wi >= a.W) continue;
-                const uint4 xv = __ldg(reinterpret_cast<const uint4*>(
-                    static_cast<const __half*>(a.x) + ((static_cast<long long>(n) * a.H + hi) * a.W + wi) * a.Cin + c0));
-                const __half* xh = reinterpret_cast<const __half*>(&xv);
+            for (int j = 0; j < kCols; j++)
+                xv[j] = __ldg(reinterpret_cast<const uint4*>(row + static_cast<long long>(min(max(wi0 + j, 0), a.W - 1)) * a.Cin));
 #pragma unroll
-                for (int j = 0; j < 8; j++) acc[j] = fmaf(__half2float(xh[j]), __half2float(wv[j * 9 + r * 3 + s]), acc[j]);
+            for (int j = 0; j < kCols; j++) {
+                const int wi = wi0 + j;
+                const float keep = (row_ok && wi >= 0 && wi < a.W) ? 1.0f : 0.0f;
+                const __half2* xh = reinterpret_cast<const __half2*>(&xv[j]);
+                float xf[8];
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    const float2 f = __half22float2(xh[e]);
+                    xf[2 * e] = f.x * keep;
+                    xf[2 * e + 1] = f.y * keep;
+                }
+#pragma unroll
+                for (int o = 0; o < kDwStrip; o++) {
+                    const int s = j - o * STRIDE;  // tap column of output o that reads input column j
+                    if (s >= 0 && s < 3) {
+#pragma unroll
+                        for (int e = 0; e < 8; e++) acc[o][e] = fmaf(xf[e], w[r * 3 + s][e], acc[o][e]);
+                    }
+                }
             }
         }
-        const long long o = ((static_cast<long long>(n) * a.Ho + ho) * a.Wo + wo) * a.Cout + c0;
-        __align__(16) __half rv[8];
-        if (a.res) *reinterpret_cast<uint4*>(rv) = __ldg(reinterpret_cast<const uint4*>(static_cast<const __half*>(a.res) + o));
-        uint4 outv;
-        uint32_t* ou = reinterpret_cast<uint32_t*>(&outv);
 #pragma unroll
-        for (int j = 0; j < 8; j += 2) {
-            float v0 = acc[j] + a.bias[c0 + j], v1 = acc[j + 1] + a.bias[c0 + j + 1];
-            if (a.res) { v0 += __half2float(rv[j]); v1 += __half2float(rv[j + 1]); }
-            ou[j / 2] = pack_half2(apply_act(v0, a.act), apply_act(v1, a.act));
+        for (int o = 0; o < kDwStrip; o++) {
+            const int wo = wo0 + o;
+            if (wo >= a.Wo) break;
+            const long long off = ((static_cast<long long>(n) * a.Ho + ho) * a.Wo + wo) * a.Cout + c0;
+            float v[8];
+#pragma unroll
+            for (int e = 0; e < 8; e++) v[e] = acc[o][e] + b[e];
+            if (res != nullptr) {
+                const uint4 rv = __ldg(reinterpret_cast<const uint4*>(res + off));
+                const __half2* rh = reinterpret_cast<const __half2*>(&rv);
+#pragma unroll
+                for (int e = 0; e < 4; e++) {
+                    const float2 f = __half22float2(rh[e]);
+                    v[2 * e] += f.x;
+                    v[2 * e + 1] += f.y;
+                }
+            }
+            uint4 outv;
+            uint32_t* ou = reinterpret_cast<uint32_t*>(&outv);
+#pragma unroll
+            for (int e = 0; e < 4; e++)
+                ou[e] = pack_half2(fminf(fmaxf(v[2 * e], lo), hi), fminf(fmaxf(v[2 * e + 1], lo), hi));
+            *reinterpret_cast<uint4*>(y + off) = outv;
         }
-        *reinterpret_cast<uint4*>(static_cast<__half*>(a.y) + o) = outv;
     }
 }
 
@@ -172,12 +231,15 @@ __global__ void __launch_bounds__(256) maxpool_kernel(const __half* x, __half* y
         const __half2 ninf = __half2half2(__ushort_as_half(0xFC00));
 #pragma unroll
         for (int j = 0; j < 4; j++) best[j] = ninf;
+        // clamped taps instead of skipped ones: a tap outside the image re-reads an in-range pixel of the
+        // same window (the maximum is unchanged) and the loads carry no branches, so they overlap
+        const int h_lo = max(ho * stride - pad, 0), h_hi = min(ho * stride - pad + k - 1, H - 1);
+        const int w_lo = max(wo * stride - pad, 0), w_hi = min(wo * stride - pad + k - 1, W - 1);
         for (int r = 0; r < k; r++) {
-            const int hi = ho * stride - pad + r;
-            if (hi < 0 || hi >= H) continue;
+            const int hi = min(max(ho * stride - pad + r, h_lo), h_hi);
+#pragma unroll 3
             for (int s = 0; s < k; s++) {
-                const int wi = wo * stride - pad + s;
-                if (wi < 0 || wi >= W) continue;
+                const int wi = min(max(wo * stride - pad + s, w_lo), w_hi);
                 const uint4 v = __ldg(reinterpret_cast<const uint4*>(x + ((static_cast<long long>(n) * H + hi) * W + wi) * C + c8 * 8));
                 const __half2* vh = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
@@ -298,9 +360,19 @@ int launch_conv_direct(const ConvArgs& a, int sm_count, cudaStream_t s) {
 
 int launch_dw3x3(const ConvArgs& a, int sm_count, cudaStream_t s) {
     if (a.kh != 3 || a.kw != 3 || a.groups != a.Cin || a.Cin != a.Cout || a.Cin % 8 || a.pool) return DLF_E_UNSUPPORTED;
-    const long long total = static_cast<long long>(a.N) * a.Ho * a.Wo * (a.Cout / 8);
+    if (a.stride != 1 && a.stride != 2) return DLF_E_UNSUPPORTED;
+    const int c8n = a.Cout / 8;
+    const int strips = (a.Wo + kDwStrip - 1) / kDwStrip;
+    const long long total = static_cast<long long>(a.N) * a.Ho * strips * c8n;
     if (total == 0) return DLF_OK;
-    dw3x3_kernel<<<grid_for((total + 255) / 256, sm_count), 256, 0, s>>>(a, total);
+    // the total thread count is a multiple of C/8: a thread keeps its channels (and its weights)
+    int step = c8n;
+    for (int d = 2; d <= 128; d *= 2)
+        if (step % 2 == 0) step /= 2;  // blocks needed for (blocks * 128) % c8n == 0: c8n / gcd(c8n, 128)
+    long long blocks = std::min<long long>((total + 127) / 128, static_cast<long long>(sm_count) * 12);
+    blocks = std::max<long long>(step, blocks / step * step);
+    if (a.stride == 1) dw3x3_kernel<1><<<static_cast<int>(blocks), 128, 0, s>>>(a, total, strips);
+    else dw3x3_kernel<2><<<static_cast<int>(blocks), 128, 0, s>>>(a, total, strips);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }

@@ -42,7 +42,11 @@ struct StemParams {
 
 __device__ __forceinline__ void work_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kWorkWarps) : "memory"); }
 
+// CIN > 0: the channel count is a compile-time constant (the tap / channel index arithmetic of the
+// gather folds away); CIN == 0: any channel count up to 4.
+template <int CIN>
 __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_constant__ CUtensorMap tmy, const StemParams p) {
+    const int cin = CIN > 0 ? CIN : p.Cin;
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t a_full_bar[2], t_full_bar[2];
     __shared__ uint32_t tmem_base_s;
@@ -77,10 +81,10 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
         reinterpret_cast<uint4*>(sbase)[i] = make_uint4(0u, 0u, 0u, 0u);
     __syncthreads();
     {
-        const int per_co = p.kh * p.kw * p.Cin;
+        const int per_co = p.kh * p.kw * cin;
         for (int i = threadIdx.x; i < p.Cout * per_co; i += kThreads) {
             const int co = i / per_co, rem = i - co * per_co;
-            const int r = rem / (p.kw * p.Cin), sc = rem - r * (p.kw * p.Cin);
+            const int r = rem / (p.kw * cin), sc = rem - r * (p.kw * cin);
             const int k = r * p.KR + sc;
             *reinterpret_cast<__half*>(bsm + (k >> 6) * 8192 + co * 128 + ((((k & 63) >> 3) ^ (co & 7)) << 4) + (k & 7) * 2) = p.w[i];
         }
@@ -111,7 +115,7 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
             }
         }
     } else {
-        const int kwc = p.kw * p.Cin;
+        const int kwc = p.kw * cin;
         const int chunks_per_row = p.KR >> 3;
         const int q = warp & 3, half = warp >> 2;
         uint32_t j = 0;
@@ -132,13 +136,13 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
                     const int hi = ho * p.stride - p.pad + r;
                     const bool row_ok = n < p.N && ho < p.Ho && wo < p.Wo && hi >= 0 && hi < p.H;
                     const int wi0 = wo * p.stride - p.pad;
-                    const __half* src = p.x + ((static_cast<long long>(n) * p.H + hi) * p.W + wi0) * p.Cin;
+                    const __half* src = p.x + ((static_cast<long long>(n) * p.H + hi) * p.W + wi0) * cin;
                     for (int ck = 0; ck < chunks_per_row; ck++) {
                         __align__(16) __half vals[8];
 #pragma unroll
                         for (int e = 0; e < 8; e++) {
                             const int idx = ck * 8 + e;               // position inside this kernel row's K slice
-                            const int wi = wi0 + idx / p.Cin;
+                            const int wi = wi0 + idx / cin;
                             const bool in = row_ok && idx < kwc && wi >= 0 && wi < p.W;
                             vals[e] = in ? src[idx] : __ushort_as_half(0);
                         }
@@ -242,7 +246,8 @@ bool stem_tc_supported(const ConvArgs& a) {
 int stem_tc_init() {
     static bool attr_set = false;
     if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(stem_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(stem_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(stem_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         if (e != cudaSuccess) return cuda_fail(e);
         attr_set = true;
     }
@@ -280,7 +285,9 @@ int launch_stem_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         if (rc) return rc;
     }
     const int grid = std::max(1, std::min(sm_count, p.n_work));
-    stem_tc_kernel<<<grid, kThreads, std::max<size_t>(smem_bytes(a), 120 * 1024), s>>>(tmy, p);
+    const size_t smem = std::max<size_t>(smem_bytes(a), 120 * 1024);
+    if (a.Cin == 3) stem_tc_kernel<3><<<grid, kThreads, smem, s>>>(tmy, p);
+    else stem_tc_kernel<0><<<grid, kThreads, smem, s>>>(tmy, p);
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
