@@ -259,6 +259,7 @@ def main():
     if args.bruteforce:
         b_ends, b_sms, _ = B.net_bruteforce(sess.net, len(layers), plans.sm_fractions(sms), 4, xd.data_ptr(),
                                             stream.cuda_stream, 2, 5)
+        sys.stderr.write("brute-force plan: ends %s sms %s\n" % (b_ends, b_sms))
         plan_list.append(("bruteforce", b_ends, b_sms))
     sampler = ClockSampler(local)
     clocks = None
@@ -341,6 +342,7 @@ def main():
                 "paper_context": "3.6x-7.9x over no-fusion/MP=1 on a Cambricon MLU100 (other hardware)"}
         if "bruteforce" in results:
             line["bruteforce"] = results["bruteforce"]
+            line["tuned_over_bruteforce"] = tuned["value"] / results["bruteforce"]["value"]
         print(json.dumps(line))
     sess.close()
     if world > 1:

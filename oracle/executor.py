@@ -189,6 +189,6 @@ def cone_outputs(layers, params, x, pixels):
         x0, x1 = max(0, px - reach), min(w, px + reach + 1)
         t = np.ascontiguousarray(x[n:n + 1, y0:y1, x0:x1, :])
         for l, p in zip(layers, params):
-            t = run_layer(l, t, p, None, 1)
+            t = run_layer(l, t, p, None, 0)
         out[j] = t[0, py - y0, px - x0, :]
     return out
