@@ -192,8 +192,11 @@ const char* dlf_net_group_kernel(const dlf_net* net, int group);
  *   DLF_OPT_CUDA_GRAPH       1 (default): dlf_net_run replays one CUDA graph that holds every
  *                               group of the plan (captured on the first run and whenever the
  *                               input / output pointers, weights, workspace or plan change);
- *                               0: launch the kernels one by one.  Does not clear the plan. */
-enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4 };
+ *                               0: launch the kernels one by one.  Does not clear the plan.
+ *   DLF_OPT_PDL              1 (default): the tensor-core kernels are launched with programmatic
+ *                               dependent launch, so that a kernel's set-up overlaps the tail of
+ *                               its predecessor; 0: plain stream order.  Process-wide. */
+enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4, DLF_OPT_PDL = 5 };
 int dlf_net_set_option(dlf_net* net, int option, int value);
 
 /* Size of the scratch array that dlf_conv_chain_run_static keeps inside the library image. */

@@ -204,6 +204,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();
+    pdl_wait();  // the set-up above overlapped the previous kernel; from here on its outputs are read
     const uint32_t tmem_base = tmem_base_s;
     const int frame_rows = p.rows * p.pitch;
 
@@ -632,8 +634,7 @@ int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int 
     }
     const int grid = std::max(1, std::min(sm_count, t.n_tiles));
     const size_t smem = std::max<size_t>(t.smem_bytes, 120 * 1024);
-    chain_tc_kernel<<<grid, kThreads, smem, s>>>(p);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_kernel(chain_tc_kernel, grid, kThreads, smem, s, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 

@@ -114,6 +114,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();
+    pdl_wait();  // everything above overlapped the previous kernel; from here on its outputs are read
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
     const int taps = p.kh * p.kw;
@@ -456,8 +458,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     }
     const int grid = std::max(1, std::min(sm_count, p.n_work));
     const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024, 120 * 1024);
-    pick_kernel(a.act, a.pool != 0, a.res != nullptr)<<<grid, kThreads, smem, s>>>(tmx, tmw, tmy, p);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_kernel(pick_kernel(a.act, a.pool != 0, a.res != nullptr), grid, kThreads, smem, s, tmx, tmw, tmy, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 

@@ -62,6 +62,24 @@ int kernels_init();
 int conv_tc_init();
 int chain_tc_init();
 
+// Launches a kernel, optionally with programmatic dependent launch (the kernel must then call
+// pdl_wait() before it touches anything its predecessor in the stream produces).
+extern int g_use_pdl;
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(static_cast<unsigned>(block));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_use_pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // kernels_mem.cu
 int launch_conv_direct(const ConvArgs& a, int sm_count, cudaStream_t s);
 int launch_dw3x3(const ConvArgs& a, int sm_count, cudaStream_t s);

@@ -27,6 +27,14 @@ __device__ __forceinline__ uint64_t global_ns() {
 #define DLF_TRACE_POINT(status, slot) do { } while (0)
 #endif
 
+// ---- programmatic dependent launch -----------------------------------------------------------------
+// A kernel launched with the programmatic-serialization attribute may start while its predecessor
+// in the stream still runs: its CTAs are scheduled as SMs free up and run their set-up (barriers,
+// TMEM allocation, bias staging); pdl_wait() then blocks until the predecessor grid has completed
+// and its memory operations are visible.  Both are no-ops for a normal launch.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---- mbarrier ---------------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");

@@ -93,6 +93,8 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
+    pdl_launch_dependents();
+    pdl_wait();  // weights are constants; the input may come from the previous kernel
     const uint32_t tmem_base = tmem_base_s;
 
     if (warp == kMmaWarp) {
@@ -286,9 +288,8 @@ int launch_stem_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     }
     const int grid = std::max(1, std::min(sm_count, p.n_work));
     const size_t smem = std::max<size_t>(smem_bytes(a), 120 * 1024);
-    if (a.Cin == 3) stem_tc_kernel<3><<<grid, kThreads, smem, s>>>(tmy, p);
-    else stem_tc_kernel<0><<<grid, kThreads, smem, s>>>(tmy, p);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = a.Cin == 3 ? launch_kernel(stem_tc_kernel<3>, grid, kThreads, smem, s, tmy, p)
+                               : launch_kernel(stem_tc_kernel<0>, grid, kThreads, smem, s, tmy, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 
