@@ -205,7 +205,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after_sync();
     pdl_launch_dependents();
-    pdl_wait();  // the set-up above overlapped the previous kernel; from here on its outputs are read
+    // the set-up above overlapped the previous kernel; from here on its outputs are read - except by the
+    // weight producers, which only read constants and may run ahead
+    if (warp < kWeightWarp0 || warp >= kInputWarp0) pdl_wait();
     const uint32_t tmem_base = tmem_base_s;
     const int frame_rows = p.rows * p.pitch;
 

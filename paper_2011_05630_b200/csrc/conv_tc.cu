@@ -115,7 +115,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     pdl_launch_dependents();
-    pdl_wait();  // everything above overlapped the previous kernel; from here on its outputs are read
+    // everything above overlapped the previous kernel; from here on its outputs are read - except by the
+    // weight producers, which only read constants and may run ahead
+    if (warp < kProdWarp0 + 2) pdl_wait();
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
     const int taps = p.kh * p.kw;
@@ -280,7 +282,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             }
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 6);
         }
-        if (!POOL && lane == 0) tma_store_wait_all();
+        if (!POOL && lane == 0) tma_store_wait_read();  // the staging tile must outlive the stores' reads; the grid's
+                                                        // completion makes their writes visible
     }
 
     tc_fence_before_sync();

@@ -202,7 +202,7 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
             if (!have) break;
             prev_t = t;
         }
-        if (threadIdx.x == 0) tma_store_wait_all();
+        if (threadIdx.x == 0) tma_store_wait_read();
     }
 
     tc_fence_before_sync();
