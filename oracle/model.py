@@ -122,11 +122,13 @@ def layer_mp(c, op_count, p):
 
 # ---- Algorithm 1 ----------------------------------------------------------------------
 
-def algorithm1(kinds, channels, ops, p, must_close_after=None):
+def algorithm1(kinds, channels, ops, p, must_close_after=None, may_close=None):
     """kinds[i]: True when layer i is a convolution / fully connected layer; channels[i],
     ops[i]: its C and operation count (ignored otherwise).  p: dict with alpha, beta,
     kappa, kappa0, s_max, op_critical.  must_close_after(start, i) -> bool forces the block
-    that started at `start` to end at layer i.  Returns (partition_index, mp_of_block)."""
+    that started at `start` to end at layer i; may_close(start, i) -> bool says whether the layers
+    start..i already form a block that can run (a block whose layers are only the beginning of a
+    fusable pattern keeps growing past the threshold).  Returns (partition_index, mp_of_block)."""
     n = len(kinds)
     partition, mp_of_block = [], []
     sum_op, sum_mp, block_size, start = 0.0, 0.0, 0, 0
@@ -139,7 +141,8 @@ def algorithm1(kinds, channels, ops, p, must_close_after=None):
         forced = (i == n - 1) or (must_close_after is not None and must_close_after(start, i))
         if block_size > 0:
             avg_mp = sum_mp / block_size
-            if sum_op / avg_mp >= p["op_critical"] or forced:
+            closable = may_close is None or may_close(start, i)
+            if (sum_op / avg_mp >= p["op_critical"] and closable) or forced:
                 partition.append(i)
                 mp = 2 ** int(math.floor(math.log2(avg_mp)))
                 if avg_mp >= p["s_max"]:  # the top step is the whole chip (32 of 32 cores in the paper)

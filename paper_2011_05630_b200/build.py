@@ -13,7 +13,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libdlfusion.so")
-SOURCES = ["api.cu", "kernels_mem.cu", "conv_tc.cu", "chain_tc.cu", "stem_tc.cu", "static_entry.cu"]
+SOURCES = ["api.cu", "kernels_mem.cu", "conv_tc.cu", "chain_tc.cu", "stem_tc.cu", "mbconv_tc.cu", "static_entry.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr"]
 

@@ -59,8 +59,8 @@ int encode_tmap(void* out_map, const void* base, int rank, const uint64_t* dims,
     return DLF_OK;
 }
 
-enum Kind { K_CHAIN_TC, K_CONV_TC, K_CONV_DIRECT, K_DW, K_FC, K_MAXPOOL, K_GAVG, K_STEM_TC };
-static const char* kKindName[] = {"chain_tc", "conv_tc", "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool", "stem_tc"};
+enum Kind { K_CHAIN_TC, K_CONV_TC, K_CONV_DIRECT, K_DW, K_FC, K_MAXPOOL, K_GAVG, K_STEM_TC, K_MBCONV };
+static const char* kKindName[] = {"chain_tc", "conv_tc", "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool", "stem_tc", "mbconv_tc"};
 
 struct Layer {
     dlf_layer_desc d;
@@ -76,6 +76,7 @@ struct Group {
     int first, last, sms;
     Kind kind;
     ChainTiling tiling;
+    MbconvTiling mb_tiling;
 };
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -168,6 +169,58 @@ static bool span_is_chain(const dlf_net* net, int first, int last) {
     return true;
 }
 
+// ---- inverted-residual pattern ------------------------------------------------------------------------
+// [1x1 conv (expansion), depthwise 3x3, 1x1 conv (projection)] or, without expansion, [depthwise 3x3,
+// 1x1 conv]: each layer reads its predecessor, no pooling, a residual only on the projection and
+// from outside the span, the maps between the layers used nowhere else.  `prefix` accepts the
+// pattern's first layers (a block that may still grow into the pattern).
+static bool pointwise_ok(const dlf_layer_desc& d) {
+    return d.op == DLF_CONV && d.groups == 1 && d.kh == 1 && d.kw == 1 && d.stride == 1 && d.pad == 0 && d.pool == 0;
+}
+static bool depthwise_ok(const dlf_layer_desc& d) {
+    return d.op == DLF_DWCONV && d.kh == 3 && d.kw == 3 && d.pad == 1 && (d.stride == 1 || d.stride == 2) && d.pool == 0 &&
+           d.res_src == -2;
+}
+static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix) {
+    const int len = last - first + 1;
+    if (len < 2 || len > 3) return false;
+    const dlf_layer_desc& d0 = net->layers[first].d;
+    const bool has_expand = d0.op == DLF_CONV;
+    const int n_full = has_expand ? 3 : 2;
+    if (len > n_full || (!prefix && len != n_full)) return false;
+    int idx = first;
+    if (has_expand) {
+        if (!pointwise_ok(d0) || d0.res_src != -2) return false;
+        idx++;
+    }
+    const dlf_layer_desc& dd = net->layers[idx].d;
+    if (!depthwise_ok(dd) || (idx > first && dd.src != idx - 1)) return false;
+    int hid = dd.cin, cout = 8;  // no projection yet (a prefix): nothing to check on its width
+    if (idx < last) {
+        const dlf_layer_desc& dp = net->layers[idx + 1].d;
+        if (!pointwise_ok(dp) || dp.src != idx || dp.res_src >= first) return false;
+        cout = dp.cout;
+    }
+    MbconvArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.N = 1; a.H = 8; a.W = 8;
+    a.Cin = has_expand ? d0.cin : hid; a.hid = hid; a.Cout = cout; a.stride = dd.stride; a.has_expand = has_expand ? 1 : 0;
+    if (!mbconv_supported(a)) return false;
+    // the maps between the layers are used nowhere else
+    const int n = static_cast<int>(net->layers.size());
+    for (int j = first + 1; j < n; j++) {
+        const dlf_layer_desc& d = net->layers[j].d;
+        const int refs[2] = {d.src, d.res_src};
+        for (int k = 0; k < 2; k++) {
+            const int r = refs[k];
+            if (r < first || r >= last) continue;
+            if (k == 0 && j <= last && r == j - 1) continue;
+            return false;
+        }
+    }
+    return true;
+}
+
 static inline const uint8_t* slot(const dlf_net* net, int idx) {
     return net->ws ? net->ws + net->layers[idx].off : nullptr;
 }
@@ -213,6 +266,26 @@ static ConvArgs conv_args(const dlf_net* net, int i, const void* in_dev, void* o
     return a;
 }
 
+static MbconvArgs mbconv_args(const dlf_net* net, int first, int last, const void* in_dev, void* out_dev) {
+    MbconvArgs a;
+    std::memset(&a, 0, sizeof(a));
+    const Layer& f = net->layers[first];
+    const Layer& z = net->layers[last];
+    const bool has_expand = f.d.op == DLF_CONV;
+    const Layer& dwl = net->layers[has_expand ? first + 1 : first];
+    a.x = f.d.src < 0 ? in_dev : slot(net, f.d.src);
+    a.w1 = has_expand ? f.w : nullptr; a.b1 = has_expand ? f.bias : nullptr;
+    a.wd = dwl.w; a.bd = dwl.bias;
+    a.w2 = z.w; a.b2 = z.bias;
+    a.res = z.d.res_src == -2 ? nullptr : (z.d.res_src < 0 ? in_dev : slot(net, z.d.res_src));
+    a.y = out_dev;
+    a.N = static_cast<int>(f.in[0]); a.H = static_cast<int>(f.in[1]); a.W = static_cast<int>(f.in[2]);
+    a.Cin = f.d.cin; a.hid = dwl.d.cin; a.Cout = z.d.cout; a.stride = dwl.d.stride;
+    a.has_expand = has_expand ? 1 : 0;
+    a.act1 = has_expand ? f.d.act : 0; a.act2 = dwl.d.act; a.act3 = z.d.act;
+    return a;
+}
+
 static bool single_kind(const dlf_net* net, int i, Kind* kind) {
     const Layer& l = net->layers[i];
     switch (l.d.op) {
@@ -248,6 +321,7 @@ static bool single_kind(const dlf_net* net, int i, Kind* kind) {
 static bool make_group(const dlf_net* net, int first, int last, int sms, Group* g) {
     g->first = first; g->last = last; g->sms = sms;
     g->tiling = ChainTiling{};
+    g->mb_tiling = MbconvTiling{};
     if (first == last) {
         // A single stride-1 3x3 layer with few channels re-reads its input nine times through the
         // per-tap kernel; the fused-chain kernel loads the tile once (measured faster up to 64 channels).
@@ -255,7 +329,13 @@ static bool make_group(const dlf_net* net, int first, int last, int sms, Group* 
         const bool prefer_chain = net->opt_single_chain || (d.op == DLF_CONV && d.kh == 3 && d.cin <= 64 && d.cout <= 64);
         if (!(prefer_chain && !net->opt_no_tc && span_is_chain(net, first, last))) return single_kind(net, first, &g->kind);
     }
-    if (net->opt_no_tc || !span_is_chain(net, first, last)) return false;
+    if (net->opt_no_tc) return false;
+    if (first < last && span_is_mbconv(net, first, last, false)) {
+        g->mb_tiling = mbconv_tiling(mbconv_args(net, first, last, nullptr, nullptr), sms);
+        g->kind = K_MBCONV;
+        return g->mb_tiling.ok;
+    }
+    if (!span_is_chain(net, first, last)) return false;
     ChainArgs a = chain_args(net, first, last, nullptr, nullptr);
     g->tiling = chain_tc_tiling(a, sms, net->dev_sms);
     g->kind = K_CHAIN_TC;
@@ -273,6 +353,7 @@ static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* 
             ChainArgs a = chain_args(net, g.first, g.last, in_dev, y);
             return launch_chain_tc(a, g.tiling, g.sms, net->opt_base_offset, status, s);
         }
+        case K_MBCONV: return launch_mbconv_tc(mbconv_args(net, g.first, g.last, in_dev, y), g.mb_tiling, g.sms, status, s);
         case K_CONV_TC: return launch_conv_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
         case K_STEM_TC: return launch_stem_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
         case K_CONV_DIRECT: return launch_conv_direct(conv_args(net, g.first, in_dev, y), g.sms, s);
@@ -301,6 +382,7 @@ namespace dlf {
 int kernels_init() {
     int rc = conv_tc_init();
     if (rc == DLF_OK) rc = chain_tc_init();
+    if (rc == DLF_OK) rc = mbconv_tc_init();
     return rc ? rc : stem_tc_init();
 }
 
@@ -642,19 +724,30 @@ int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_
             sum_mp += layer_sms(l, *params, s_max);
             block++;
         }
-        bool forced = (i == n - 1) || !span_is_chain(net, start, i + 1);
+        // a block may grow while its layers are, or can still become, a group one kernel runs; it may
+        // close only where they already are one (inside an inverted-residual block it keeps growing)
+        bool forced = (i == n - 1) || !(span_is_chain(net, start, i + 1) || span_is_mbconv(net, start, i + 1, true));
+        const bool closable = (i == start) || span_is_chain(net, start, i) || span_is_mbconv(net, start, i, false);
         if (!forced && params->legalise) {
             Group g;
-            forced = !make_group(net, start, i + 1, s_max, &g);
+            if (i + 1 > start && (span_is_chain(net, start, i + 1) || span_is_mbconv(net, start, i + 1, false)))
+                forced = !make_group(net, start, i + 1, s_max, &g);
         }
         if (block > 0) {
             const double avg = sum_mp / block;
-            if (sum_op / avg >= params->op_critical || forced) {
-                group_end[ng] = i;
+            if ((sum_op / avg >= params->op_critical && closable) || forced) {
                 int mp = 1 << static_cast<int>(std::floor(std::log2(avg)));
                 if (avg >= s_max) mp = s_max;  // the top step is the whole chip, as 32 of 32 cores in the paper
-                sm_count[ng] = std::min(std::max(mp, 1), s_max);
-                ng++;
+                mp = std::min(std::max(mp, 1), s_max);
+                Group g;
+                if (params->legalise && i > start && !make_group(net, start, i, mp, &g)) {
+                    // the block cannot run as one kernel: one group per layer
+                    for (int j = start; j <= i; j++) { group_end[ng] = j; sm_count[ng] = mp; ng++; }
+                } else {
+                    group_end[ng] = i;
+                    sm_count[ng] = mp;
+                    ng++;
+                }
                 sum_op = sum_mp = 0.0;
                 block = 0;
                 start = i + 1;
@@ -898,7 +991,7 @@ int dlf_net_group_model(const dlf_net* net, int group, int64_t* flops, int64_t* 
     }
     if (flops) *flops = fl;
     if (hbm_bytes) *hbm_bytes = by;
-    if (redundancy) *redundancy = g.kind == K_CHAIN_TC ? g.tiling.redundancy : 1.0;
+    if (redundancy) *redundancy = g.kind == K_CHAIN_TC ? g.tiling.redundancy : (g.kind == K_MBCONV ? g.mb_tiling.redundancy : 1.0);
     if (launches) *launches = 1;
     return DLF_OK;
 }

@@ -99,6 +99,27 @@ bool stem_tc_supported(const ConvArgs& a);
 int stem_tc_init();
 int launch_stem_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s);
 
+// mbconv_tc.cu: fused inverted-residual block (1x1 expansion, depthwise 3x3, 1x1 projection)
+struct MbconvArgs {
+    const void* x;           // [N][H][W][Cin]
+    const void *w1, *wd, *w2;  // [hid][Cin], [hid][3][3][1], [Cout][hid]
+    const float *b1, *bd, *b2;
+    const void* res;         // [N][Ho][Wo][Cout] or null
+    void* y;
+    int N, H, W, Cin, hid, Cout, stride;
+    int has_expand, act1, act2, act3;
+};
+struct MbconvTiling {
+    int th, tw, fh, fw, nb1, nb2, tiles_h, tiles_w, n_tiles, stages, stage_bytes;
+    size_t smem_bytes;
+    double redundancy;
+    bool ok;
+};
+bool mbconv_supported(const MbconvArgs& a);
+MbconvTiling mbconv_tiling(const MbconvArgs& a, int sm_count);
+int mbconv_tc_init();
+int launch_mbconv_tc(const MbconvArgs& a, const MbconvTiling& t, int sm_count, int* status_dev, cudaStream_t s);
+
 // chain_tc.cu
 ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms);
 int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int base_offset_mode, int* status_dev,

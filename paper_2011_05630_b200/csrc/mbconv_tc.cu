@@ -1,0 +1,494 @@
+// Fused inverted-residual block (MobileNetV2): 1x1 expansion (+bias, activation) -> depthwise 3x3,
+// stride 1 or 2 (+bias, activation) -> 1x1 projection (+bias, optional residual, activation), as ONE
+// kernel.  The expanded map (6x the block's input, the dominant HBM traffic of the unfused plan)
+// never exists in memory: the hidden dimension is processed in chunks of 64 channels.  Per output
+// tile and chunk:
+//   1. expansion on the tensor cores: D1[frame rows x 64] = X[frame rows x C_in] * W1[chunk]^T, the
+//      input frame (tile + 1-pixel halo, TMA-loaded once per tile) staying in shared memory;
+//   2. epilogue 1 (CUDA cores): bias, activation, fp16 rounding, zero outside the image (the
+//      depthwise layer's padding) -> hidden tile H in shared memory;
+//   3. depthwise 3x3 on the CUDA cores (exact per channel, so chunking the hidden dimension changes
+//      nothing): nine 128-bit shared-memory reads per 8 channels, fp32 accumulate, bias, activation,
+//      fp16 rounding -> tile Hd, laid out as the next GEMM's operand;
+//   4. projection on the tensor cores: D2[tile rows x C_out] += Hd * W2[:, chunk]^T, accumulated in
+//      tensor memory across the chunks (fp32, the same sum as the unchunked layer);
+// then epilogue 2: bias, residual, activation, fp16 rounding, global store.  Every intermediate is
+// rounded to fp16 exactly where the layer-by-layer execution rounds it.  Without an expansion layer
+// (the network's first block) steps 1-2 are skipped and the depthwise layer reads the input frame.
+//
+// Warps: 0-7 work (epilogues and depthwise), 8 UMMA issuer, 9 input producer, 10-11 weight producers.
+#include <cuda.h>
+#include <cuda_fp16.h>
+
+#include <algorithm>
+#include <cstring>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace dlf {
+
+namespace {
+
+constexpr int kWorkWarps = 8;
+constexpr int kMmaWarp = kWorkWarps;
+constexpr int kInWarp = kWorkWarps + 1;
+constexpr int kW1Warp = kWorkWarps + 2;
+constexpr int kW2Warp = kWorkWarps + 3;
+constexpr int kThreads = 32 * (kWorkWarps + 4);
+constexpr int kMaxSmem = 232448 - 1024;
+constexpr int kPlane = 128 * 128;  // 128 rows x 64 channels
+
+struct MbParams {
+    CUtensorMap tmx, tmw1, tmw2;
+    int N, H, W, Cin, hid, Cout, Ho, Wo, stride;
+    int has_expand, act1, act2, act3;
+    int th, tw, fh, fw, FR, nb1, nb2;   // output tile, input frame, frame rows, 128-row blocks of the two GEMMs
+    int tiles_h, tiles_w, n_tiles;
+    int kin, chunks, n2_pad;            // 64-channel planes of the input, hidden chunks, C_out rounded up to 16
+    int ksteps_in_last;
+    int x_off, h_off, hd_off, ring_off, stage_bytes, stages, dw_off, bias_off;  // shared-memory byte offsets
+    int d2_col;                         // first TMEM column of the projection accumulator
+    int w2_off, n_split, n_each;        // projection slab inside a ring stage; C_out > 256 is issued as two halves
+    const __half* wd;
+    const float *b1, *bd, *b2;
+    const __half* res;
+    __half* out;
+    int* status;
+};
+
+__device__ __forceinline__ void work_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kWorkWarps) : "memory"); }
+
+__device__ __forceinline__ float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi); }
+
+__global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_constant__ MbParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t x_full, x_empty, w_full[4], w_empty[4], d1_full, d1_free, hd_ready, hd_free, d2_full, d2_free;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sb = smem_raw + (base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    volatile int* abort_flag = &abort_s;
+    float* dw_s = reinterpret_cast<float*>(sb + p.dw_off);      // [9][64] depthwise weights of the chunk, then [64] bias
+    float* bias_s = reinterpret_cast<float*>(sb + p.bias_off);  // b1[chunks * 64] then b2[n2_pad]
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        mbar_init(&x_full, 1);
+        mbar_init(&x_empty, p.has_expand ? 1 : kWorkWarps);
+        for (int i = 0; i < p.stages; i++) {
+            mbar_init(&w_full[i], p.has_expand ? 2 : 1);
+            mbar_init(&w_empty[i], 1);
+        }
+        mbar_init(&d1_full, 1);
+        mbar_init(&d1_free, kWorkWarps);
+        mbar_init(&hd_ready, kWorkWarps);
+        mbar_init(&hd_free, 1);
+        mbar_init(&d2_full, 1);
+        mbar_init(&d2_free, kWorkWarps);
+        fence_barrier_init();
+        tma_prefetch_desc(&p.tmx);
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(&tmem_base_s, 512);
+        tmem_relinquish();
+    }
+    for (int i = threadIdx.x; i < p.chunks * 64; i += kThreads) bias_s[i] = (p.has_expand && i < p.hid) ? __ldg(p.b1 + i) : 0.0f;
+    for (int i = threadIdx.x; i < p.n2_pad; i += kThreads) bias_s[p.chunks * 64 + i] = i < p.Cout ? __ldg(p.b2 + i) : 0.0f;
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    pdl_launch_dependents();
+    if (warp != kW1Warp && warp != kW2Warp) pdl_wait();  // the weight producers only read constants
+    const uint32_t tmem_base = tmem_base_s;
+
+    if (warp == kInWarp) {
+        // ---- input producer: the tile's frame, one box per 64-channel plane ---------------------------
+        if (lane == 0) {
+            uint32_t ti = 0;
+            for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x, ti++) {
+                const int txi = t % p.tiles_w, tyi = (t / p.tiles_w) % p.tiles_h, n = t / (p.tiles_w * p.tiles_h);
+                if (!mbar_wait(&x_empty, (ti & 1u) ^ 1u, abort_flag, p.status, 0xB00 | (blockIdx.x << 12))) break;
+                mbar_expect_tx(&x_full, static_cast<uint32_t>(p.kin) * p.FR * 128u);
+                for (int pl = 0; pl < p.kin; pl++)
+                    tma_load_4d(sb + p.x_off + pl * p.nb1 * kPlane, &p.tmx, &x_full, pl * 64, txi * p.tw * p.stride - 1,
+                                tyi * p.th * p.stride - 1, n);
+            }
+        }
+    } else if (warp == kW1Warp || warp == kW2Warp) {
+        // ---- weight producers: per chunk the expansion slab [64 hidden][C_in] and the projection
+        //      slab [C_out][64 hidden]; one ring stage holds both ---------------------------------------
+        if (lane == 0 && (warp == kW2Warp || p.has_expand)) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x)
+                for (int hc = 0; hc < p.chunks; hc++, it++) {
+                    const int st = it % p.stages;
+                    ok = mbar_wait(&w_empty[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status, 0xC00 | (blockIdx.x << 12));
+                    if (!ok) break;
+                    uint8_t* dst = sb + p.ring_off + st * p.stage_bytes;
+                    if (warp == kW1Warp) {
+                        mbar_expect_tx(&w_full[st], static_cast<uint32_t>(p.kin) * 8192u);
+                        for (int pl = 0; pl < p.kin; pl++) tma_load_3d(dst + pl * 8192, &p.tmw1, &w_full[st], pl * 64, hc * 64, 0);
+                    } else {
+                        mbar_expect_tx(&w_full[st], static_cast<uint32_t>(p.n2_pad) * 128u);
+                        for (int j = 0; j < p.n_split; j++)
+                            tma_load_3d(dst + p.w2_off + j * p.n_each * 128, &p.tmw2, &w_full[st], hc * 64, j * p.n_each, 0);
+                    }
+                }
+        }
+    } else if (warp == kMmaWarp) {
+        // ---- UMMA issuer -------------------------------------------------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc1 = umma_idesc_f16(64), idesc2 = umma_idesc_f16(p.n_each);
+            uint32_t ti = 0, cc = 0;  // tiles and chunks done so far (barrier phases)
+            bool ok = true;
+            auto issue_expand = [&](uint32_t chunk_index) {
+                // D1 = X * W1[chunk]^T over the input planes
+                const int st = chunk_index % p.stages;
+                const uint32_t wsm = base + p.ring_off + st * p.stage_bytes;
+                for (int pl = 0; pl < p.kin; pl++) {
+                    const int ksteps = (pl == p.kin - 1) ? p.ksteps_in_last : 4;
+                    const uint32_t b_lo = umma_desc_lo(wsm + pl * 8192);
+                    for (int b = 0; b < p.nb1; b++) {
+                        const uint32_t a_lo = umma_desc_lo(base + p.x_off + (pl * p.nb1 + b) * kPlane);
+                        for (int ks = 0; ks < ksteps; ks++)
+                            umma_f16_lo(tmem_base + b * 64u, a_lo + 2 * ks, kDescHiSw128, b_lo + 2 * ks, idesc1, (pl | ks) != 0);
+                    }
+                }
+                umma_commit(&d1_full);
+            };
+            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x, ti++) {
+                ok = mbar_wait(&x_full, ti & 1u, abort_flag, p.status, 0xD00 | (blockIdx.x << 12));
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (p.has_expand) {
+                    ok = mbar_wait(&w_full[cc % p.stages], (cc / p.stages) & 1u, abort_flag, p.status, 0xD10 | (blockIdx.x << 12));
+                    if (ok && cc > 0) ok = mbar_wait(&d1_free, (cc - 1) & 1u, abort_flag, p.status, 0xD20 | (blockIdx.x << 12));
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_expand(cc);
+                }
+                for (int hc = 0; hc < p.chunks && ok; hc++, cc++) {
+                    if (p.has_expand && hc + 1 < p.chunks) {
+                        // the next chunk's expansion overlaps this chunk's depthwise step
+                        ok = mbar_wait(&w_full[(cc + 1) % p.stages], ((cc + 1) / p.stages) & 1u, abort_flag, p.status, 0xD30 | (blockIdx.x << 12));
+                        if (ok) ok = mbar_wait(&d1_free, cc & 1u, abort_flag, p.status, 0xD40 | (blockIdx.x << 12));
+                        if (!ok) break;
+                        tc_fence_after_sync();
+                        issue_expand(cc + 1);
+                    } else if (!p.has_expand) {
+                        ok = mbar_wait(&w_full[cc % p.stages], (cc / p.stages) & 1u, abort_flag, p.status, 0xD50 | (blockIdx.x << 12));
+                        if (!ok) break;
+                    }
+                    if (p.has_expand && hc + 1 == p.chunks) umma_commit(&x_empty);  // the frame is read by the expansions only
+                    // projection of this chunk once its depthwise tile is in shared memory
+                    ok = mbar_wait(&hd_ready, cc & 1u, abort_flag, p.status, 0xD60 | (blockIdx.x << 12));
+                    if (ok && hc == 0 && ti > 0) ok = mbar_wait(&d2_free, (ti - 1) & 1u, abort_flag, p.status, 0xD70 | (blockIdx.x << 12));
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const int st = cc % p.stages;
+                    for (int j = 0; j < p.n_split; j++) {
+                        const uint32_t b_lo = umma_desc_lo(base + p.ring_off + st * p.stage_bytes + p.w2_off + j * p.n_each * 128);
+                        for (int b = 0; b < p.nb2; b++) {
+                            const uint32_t a_lo = umma_desc_lo(base + p.hd_off + b * kPlane);
+                            for (int ks = 0; ks < 4; ks++)
+                                umma_f16_lo(tmem_base + p.d2_col + b * p.n2_pad + j * p.n_each, a_lo + 2 * ks, kDescHiSw128, b_lo + 2 * ks,
+                                            idesc2, (hc | ks) != 0);
+                        }
+                    }
+                    umma_commit(&hd_free);
+                    umma_commit(&w_empty[st]);
+                    if (hc + 1 == p.chunks) umma_commit(&d2_full);
+                }
+            }
+        }
+    } else {
+        // ---- work warps: epilogue 1, depthwise, epilogue 2 ---------------------------------------------------
+        const int wt = threadIdx.x;  // 0..255
+        const int q = warp & 3, half = warp >> 2;
+        const float lo1 = p.act1 >= 1 ? 0.0f : -INFINITY, hi1 = p.act1 == 2 ? 6.0f : INFINITY;
+        const float lo2 = p.act2 >= 1 ? 0.0f : -INFINITY, hi2 = p.act2 == 2 ? 6.0f : INFINITY;
+        const float lo3 = p.act3 >= 1 ? 0.0f : -INFINITY, hi3 = p.act3 == 2 ? 6.0f : INFINITY;
+        uint8_t* hbuf = sb + (p.has_expand ? p.h_off : p.x_off);
+        uint8_t* hdbuf = sb + p.hd_off;
+        uint32_t ti = 0, cc = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x, ti++) {
+            const int txi = t % p.tiles_w, tyi = (t / p.tiles_w) % p.tiles_h, n = t / (p.tiles_w * p.tiles_h);
+            const int oy0 = tyi * p.th, ox0 = txi * p.tw;
+            const int iy0 = oy0 * p.stride - 1, ix0 = ox0 * p.stride - 1;
+            if (!p.has_expand) {
+                ok = mbar_wait(&x_full, ti & 1u, abort_flag, p.status, 0xE00 | (blockIdx.x << 12));
+                if (!ok) break;
+            }
+            for (int hc = 0; hc < p.chunks && ok; hc++, cc++) {
+                // depthwise weights and bias of the chunk (channels past `hid` are zero)
+                for (int i = wt; i < 640; i += 32 * kWorkWarps) {
+                    const int ch = hc * 64 + (i & 63), tap = i >> 6;
+                    float v = 0.0f;
+                    if (ch < p.hid) v = tap < 9 ? __half2float(__ldg(p.wd + ch * 9 + tap)) : __ldg(p.bd + ch);
+                    dw_s[i] = v;
+                }
+                if (p.has_expand) {
+                    // ---- epilogue 1: D1 -> H (fp16, zero outside the image) ------------------------------
+                    ok = mbar_wait(&d1_full, cc & 1u, abort_flag, p.status, 0xE10 | (blockIdx.x << 12));
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    for (int b = 0; b < p.nb1; b++) {
+                        const int r = b * 128 + q * 32 + lane;
+                        const int fy = r / p.fw, fx = r - fy * p.fw;
+                        const int gy = iy0 + fy, gx = ix0 + fx;
+                        const bool in_img = r < p.FR && gy >= 0 && gy < p.H && gx >= 0 && gx < p.W;
+                        float v[32];
+                        __syncwarp();
+                        tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 64u + half * 32u, v);
+                        if (r < p.FR) {
+                            const float* bb = bias_s + hc * 64 + half * 32;
+#pragma unroll
+                            for (int g = 0; g < 4; g++) {
+                                uint4 val = make_uint4(0u, 0u, 0u, 0u);
+                                if (in_img) {
+                                    val.x = pack_half2(clampf(v[g * 8 + 0] + bb[g * 8 + 0], lo1, hi1), clampf(v[g * 8 + 1] + bb[g * 8 + 1], lo1, hi1));
+                                    val.y = pack_half2(clampf(v[g * 8 + 2] + bb[g * 8 + 2], lo1, hi1), clampf(v[g * 8 + 3] + bb[g * 8 + 3], lo1, hi1));
+                                    val.z = pack_half2(clampf(v[g * 8 + 4] + bb[g * 8 + 4], lo1, hi1), clampf(v[g * 8 + 5] + bb[g * 8 + 5], lo1, hi1));
+                                    val.w = pack_half2(clampf(v[g * 8 + 6] + bb[g * 8 + 6], lo1, hi1), clampf(v[g * 8 + 7] + bb[g * 8 + 7], lo1, hi1));
+                                }
+                                const int g8 = half * 4 + g;
+                                *reinterpret_cast<uint4*>(hbuf + r * 128 + ((g8 ^ (r & 7)) << 4)) = val;
+                            }
+                        }
+                    }
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&d1_free);
+                }
+                work_bar_sync();  // H (and the depthwise weights) complete
+                if (cc > 0) {
+                    ok = mbar_wait(&hd_free, (cc - 1) & 1u, abort_flag, p.status, 0xE20 | (blockIdx.x << 12));
+                    if (!ok) break;
+                }
+                // ---- depthwise 3x3: H -> Hd ---------------------------------------------------------------
+                const uint8_t* hsrc = hbuf + (p.has_expand ? 0 : hc * p.nb1 * kPlane);
+                for (int item = wt; item < p.th * p.tw * 8; item += 32 * kWorkWarps) {
+                    const int g8 = item & 7, o = item >> 3;
+                    const int oy = o / p.tw, ox = o - oy * p.tw;
+                    float acc[8];
+#pragma unroll
+                    for (int e = 0; e < 8; e++) acc[e] = 0.0f;
+#pragma unroll
+                    for (int r = 0; r < 3; r++)
+#pragma unroll
+                        for (int c = 0; c < 3; c++) {
+                            const int qrow = (oy * p.stride + r) * p.fw + ox * p.stride + c;
+                            const uint4 xv = *reinterpret_cast<const uint4*>(hsrc + qrow * 128 + ((g8 ^ (qrow & 7)) << 4));
+                            const __half2* xh = reinterpret_cast<const __half2*>(&xv);
+                            const float* wv = dw_s + (r * 3 + c) * 64 + g8 * 8;
+#pragma unroll
+                            for (int e = 0; e < 4; e++) {
+                                const float2 f = __half22float2(xh[e]);
+                                acc[2 * e] = fmaf(f.x, wv[2 * e], acc[2 * e]);
+                                acc[2 * e + 1] = fmaf(f.y, wv[2 * e + 1], acc[2 * e + 1]);
+                            }
+                        }
+                    const float* bv = dw_s + 576 + g8 * 8;
+                    uint4 val;
+                    val.x = pack_half2(clampf(acc[0] + bv[0], lo2, hi2), clampf(acc[1] + bv[1], lo2, hi2));
+                    val.y = pack_half2(clampf(acc[2] + bv[2], lo2, hi2), clampf(acc[3] + bv[3], lo2, hi2));
+                    val.z = pack_half2(clampf(acc[4] + bv[4], lo2, hi2), clampf(acc[5] + bv[5], lo2, hi2));
+                    val.w = pack_half2(clampf(acc[6] + bv[6], lo2, hi2), clampf(acc[7] + bv[7], lo2, hi2));
+                    *reinterpret_cast<uint4*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4)) = val;
+                }
+                fence_proxy_async_smem();  // the projection UMMAs read Hd through the async proxy
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&hd_ready);
+                if (!p.has_expand && hc + 1 == p.chunks && lane == 0) mbar_arrive(&x_empty);
+                work_bar_sync();  // nobody still reads H / the depthwise weights when the next chunk overwrites them
+            }
+            if (!ok) break;
+            // ---- epilogue 2: D2 -> global -------------------------------------------------------------------
+            ok = mbar_wait(&d2_full, ti & 1u, abort_flag, p.status, 0xE30 | (blockIdx.x << 12));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const float* b2s = bias_s + p.chunks * 64;
+            for (int b = 0; b < p.nb2; b++) {
+                const int o = b * 128 + q * 32 + lane;
+                const int oy = o / p.tw, ox = o - oy * p.tw;
+                const int gy = oy0 + oy, gx = ox0 + ox;
+                const bool live = o < p.th * p.tw && gy < p.Ho && gx < p.Wo;
+                const long long gpix = (static_cast<long long>(n) * p.Ho + gy) * p.Wo + gx;
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + p.d2_col + b * p.n2_pad;
+                for (int c0 = half * 16; c0 < p.n2_pad; c0 += 32) {
+                    float v[16];
+                    __syncwarp();
+                    tmem_ld16(taddr + c0, v);
+                    if (!live) continue;
+#pragma unroll
+                    for (int g = 0; g < 2; g++) {
+                        const int co = c0 + g * 8;
+                        if (co >= p.Cout) break;
+                        float a[8];
+#pragma unroll
+                        for (int e = 0; e < 8; e++) a[e] = v[g * 8 + e] + b2s[co + e];
+                        if (p.res != nullptr) {
+                            const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.res + gpix * p.Cout + co));
+                            const __half2* rh = reinterpret_cast<const __half2*>(&rv);
+#pragma unroll
+                            for (int e = 0; e < 4; e++) {
+                                const float2 f = __half22float2(rh[e]);
+                                a[2 * e] += f.x;
+                                a[2 * e + 1] += f.y;
+                            }
+                        }
+                        uint4 val;
+                        val.x = pack_half2(clampf(a[0], lo3, hi3), clampf(a[1], lo3, hi3));
+                        val.y = pack_half2(clampf(a[2], lo3, hi3), clampf(a[3], lo3, hi3));
+                        val.z = pack_half2(clampf(a[4], lo3, hi3), clampf(a[5], lo3, hi3));
+                        val.w = pack_half2(clampf(a[6], lo3, hi3), clampf(a[7], lo3, hi3));
+                        *reinterpret_cast<uint4*>(p.out + gpix * p.Cout + co) = val;
+                    }
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&d2_free);
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == kMmaWarp) {
+        if (abort_s) __nanosleep(20000);
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
+    }
+}
+
+int pad16(int c) { return (c + 15) / 16 * 16; }
+
+}  // namespace
+
+bool mbconv_supported(const MbconvArgs& a) {
+    if (a.Cin % 8 || a.hid % 16 || a.Cout % 8 || a.Cin > 256 || a.Cout > 512 || a.hid > 1024) return false;
+    if (pad16(a.Cout) > 256 && pad16(a.Cout) % 32) return false;  // issued as two equal halves
+    if (a.stride != 1 && a.stride != 2) return false;
+    if (!a.has_expand && a.hid != a.Cin) return false;
+    return a.N >= 1 && a.H >= 1 && a.W >= 1;
+}
+
+// Output tile of the fused block from the SM count: candidates whose buffers and accumulators fit,
+// least (waves x per-tile work).
+MbconvTiling mbconv_tiling(const MbconvArgs& a, int sm_count) {
+    MbconvTiling best{};
+    best.ok = false;
+    if (!mbconv_supported(a) || sm_count < 1) return best;
+    const int Ho = (a.H + 2 - 3) / a.stride + 1, Wo = (a.W + 2 - 3) / a.stride + 1;
+    const int kin = (a.Cin + 63) / 64, chunks = (a.hid + 63) / 64, n2 = pad16(a.Cout);
+    static const int cand[] = {2, 4, 7, 8, 14, 16};
+    double best_cost = -1.0;
+    for (int th : cand)
+        for (int tw : cand) {
+            if (th > std::max(Ho, 2) * 2 || tw > std::max(Wo, 2) * 2) continue;
+            const int fh = (th - 1) * a.stride + 3, fw = (tw - 1) * a.stride + 3;
+            if (fh > 256 || fw > 256) continue;
+            const int FR = fh * fw, nb1 = (FR + 127) / 128, nb2 = (th * tw + 127) / 128;
+            const int d1_cols = a.has_expand ? nb1 * 64 : 0;
+            if (d1_cols + nb2 * n2 > 512) continue;
+            const int stage = kin * 8192 * (a.has_expand ? 1 : 0) + n2 * 128;
+            const size_t fixed = static_cast<size_t>(kin) * nb1 * kPlane + (a.has_expand ? nb1 * kPlane : 0) + static_cast<size_t>(nb2) * kPlane +
+                                 4096 + static_cast<size_t>(chunks * 64 + n2) * 4 + 2048;
+            int stages = 3;
+            while (stages > 2 && fixed + static_cast<size_t>(stages) * stage > static_cast<size_t>(kMaxSmem)) stages--;
+            if (fixed + static_cast<size_t>(stages) * stage > static_cast<size_t>(kMaxSmem)) continue;
+            const int tiles_h = (Ho + th - 1) / th, tiles_w = (Wo + tw - 1) / tw;
+            const long long n_tiles = static_cast<long long>(a.N) * tiles_h * tiles_w;
+            if (n_tiles > 0x7fffffffLL) continue;
+            const long long waves = (n_tiles + sm_count - 1) / sm_count;
+            // per chunk: epilogue-1 rows + depthwise items on 256 threads, plus hand-off latency
+            const double per_chunk = (a.has_expand ? nb1 * 128 * 2.0 : 0.0) + th * tw * 8 * 6.0 + 1500.0;
+            const double cost = static_cast<double>(waves) * (chunks * per_chunk + 3000.0);
+            if (best_cost < 0 || cost < best_cost) {
+                best_cost = cost;
+                best.th = th; best.tw = tw; best.fh = fh; best.fw = fw; best.nb1 = nb1; best.nb2 = nb2;
+                best.tiles_h = tiles_h; best.tiles_w = tiles_w; best.n_tiles = static_cast<int>(n_tiles);
+                best.stages = stages; best.stage_bytes = stage;
+                best.smem_bytes = fixed + static_cast<size_t>(stages) * stage;
+                best.redundancy = static_cast<double>(FR) / (std::min(th, Ho) * a.stride * std::min(tw, Wo) * a.stride);
+                best.ok = true;
+            }
+        }
+    return best;
+}
+
+int mbconv_tc_init() {
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(mbconv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+        if (e != cudaSuccess) return cuda_fail(e);
+        attr_set = true;
+    }
+    return DLF_OK;
+}
+
+int launch_mbconv_tc(const MbconvArgs& a, const MbconvTiling& t, int sm_count, int* status_dev, cudaStream_t s) {
+    if (!t.ok) return DLF_E_PLAN;
+    int rc = mbconv_tc_init();
+    if (rc) return rc;
+    MbParams p;
+    std::memset(&p, 0, sizeof(p));
+    p.N = a.N; p.H = a.H; p.W = a.W; p.Cin = a.Cin; p.hid = a.hid; p.Cout = a.Cout; p.stride = a.stride;
+    p.Ho = (a.H + 2 - 3) / a.stride + 1; p.Wo = (a.W + 2 - 3) / a.stride + 1;
+    p.has_expand = a.has_expand; p.act1 = a.act1; p.act2 = a.act2; p.act3 = a.act3;
+    p.th = t.th; p.tw = t.tw; p.fh = t.fh; p.fw = t.fw; p.FR = t.fh * t.fw; p.nb1 = t.nb1; p.nb2 = t.nb2;
+    p.tiles_h = t.tiles_h; p.tiles_w = t.tiles_w; p.n_tiles = t.n_tiles;
+    p.kin = (a.Cin + 63) / 64; p.chunks = (a.hid + 63) / 64; p.n2_pad = pad16(a.Cout);
+    p.ksteps_in_last = ((a.Cin - (p.kin - 1) * 64) + 15) / 16;
+    p.x_off = 0;
+    p.h_off = p.kin * p.nb1 * kPlane;
+    p.hd_off = p.h_off + (a.has_expand ? p.nb1 * kPlane : 0);
+    p.ring_off = p.hd_off + p.nb2 * kPlane;
+    p.stage_bytes = t.stage_bytes; p.stages = t.stages;
+    p.dw_off = p.ring_off + p.stages * p.stage_bytes;
+    p.dw_off = (p.dw_off + 1023) / 1024 * 1024;
+    p.bias_off = p.dw_off + 4096;
+    p.d2_col = a.has_expand ? p.nb1 * 64 : 0;
+    p.w2_off = a.has_expand ? p.kin * 8192 : 0;
+    p.n_split = p.n2_pad > 256 ? 2 : 1;
+    p.n_each = p.n2_pad / p.n_split;
+    p.wd = static_cast<const __half*>(a.wd); p.b1 = a.b1; p.bd = a.bd; p.b2 = a.b2;
+    p.res = static_cast<const __half*>(a.res); p.out = static_cast<__half*>(a.y); p.status = status_dev;
+    {
+        const uint64_t dims[4] = {static_cast<uint64_t>(a.Cin), static_cast<uint64_t>(a.W), static_cast<uint64_t>(a.H), static_cast<uint64_t>(a.N)};
+        const uint64_t strides[3] = {static_cast<uint64_t>(a.Cin) * 2, static_cast<uint64_t>(a.W) * a.Cin * 2,
+                                     static_cast<uint64_t>(a.H) * a.W * a.Cin * 2};
+        const uint32_t box[4] = {64, static_cast<uint32_t>(t.fw), static_cast<uint32_t>(t.fh), 1};
+        const uint32_t es[4] = {1, 1, 1, 1};
+        rc = encode_tmap(&p.tmx, a.x, 4, dims, strides, box, es);
+        if (rc) return rc;
+    }
+    if (a.has_expand) {  // W1 [hid][C_in] seen as (C_in, hid, 1)
+        const uint64_t dims[3] = {static_cast<uint64_t>(a.Cin), static_cast<uint64_t>(a.hid), 1};
+        const uint64_t strides[2] = {static_cast<uint64_t>(a.Cin) * 2, static_cast<uint64_t>(a.hid) * a.Cin * 2};
+        const uint32_t box[3] = {64, 64, 1};
+        const uint32_t es[3] = {1, 1, 1};
+        rc = encode_tmap(&p.tmw1, a.w1, 3, dims, strides, box, es);
+        if (rc) return rc;
+    }
+    {  // W2 [C_out][hid] seen as (hid, C_out, 1)
+        const uint64_t dims[3] = {static_cast<uint64_t>(a.hid), static_cast<uint64_t>(a.Cout), 1};
+        const uint64_t strides[2] = {static_cast<uint64_t>(a.hid) * 2, static_cast<uint64_t>(a.Cout) * a.hid * 2};
+        const uint32_t box[3] = {64, static_cast<uint32_t>(p.n_each), 1};
+        const uint32_t es[3] = {1, 1, 1};
+        rc = encode_tmap(&p.tmw2, a.w2, 3, dims, strides, box, es);
+        if (rc) return rc;
+    }
+    const int grid = std::max(1, std::min(sm_count, t.n_tiles));
+    const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + (p.chunks * 64 + p.n2_pad) * 4 + 2048, 120 * 1024);
+    if (smem > static_cast<size_t>(kMaxSmem)) return DLF_E_PLAN;
+    cudaError_t e = launch_kernel(mbconv_tc_kernel, grid, kThreads, smem, s, p);
+    return e == cudaSuccess ? DLF_OK : cuda_fail(e);
+}
+
+}  // namespace dlf

@@ -34,6 +34,9 @@ def test_network_every_boundary(name, builder, batch):
     todo = [("unfused", None, None)]
     ends, smc = plans.tuned_plan(sess.net, len(layers))
     todo.append(("tuned", ends, smc))
+    if name == "mobilenet_v2":   # one group per inverted-residual block (the critical op count set out of reach)
+        ends, smc = plans.tuned_plan(sess.net, len(layers), op_critical=1e30)
+        todo.append(("block-fused", ends, smc))
     for what, e, s in todo:
         ends_now, _ = sess.set_plan(e, s)
         out = sess.run(xd).cpu().numpy()

@@ -177,3 +177,55 @@ def test_illegal_plans_are_rejected():
             B.net_set_plan(sess.net, ends, sm)
         assert e.value.status == B.E_PLAN
     G.check_plan(sess, xd, ref, [0, 1, 2], [2, 2, 2], "legal")
+
+
+# ---- fused inverted-residual blocks --------------------------------------------------------------------
+def _mbconv(cin, t, cout, stride, first):
+    """Layers of one inverted-residual block whose input is layer `first - 1` (or the network input)."""
+    hid = cin * t
+    L = []
+    if t != 1:
+        L.append(_conv(cin, hid, 1, act="relu6", src=first - 1))
+    L.append(_conv(hid, hid, 3, stride=stride, act="relu6", groups=hid, op="dwconv", src=first + len(L) - 1))
+    L.append(_conv(hid, cout, 1, act="none", src=first + len(L) - 1,
+                   res_src=(first - 1) if (stride == 1 and cin == cout) else -2))
+    return L
+
+
+MBCONV = [
+    # (n, h, w, cin, t, cout, stride)
+    (2, 16, 16, 16, 6, 24, 2),      # hidden 96 = 64 + 32
+    (2, 19, 21, 24, 6, 24, 1),      # hidden 144, residual, ragged tiles
+    (3, 14, 14, 64, 6, 64, 1),      # six hidden chunks, residual
+    (2, 15, 13, 32, 1, 16, 1),      # no expansion layer
+    (2, 7, 7, 160, 6, 320, 1),      # three input planes, projection issued as two halves
+    (1, 28, 28, 32, 6, 64, 2),
+]
+
+
+@pytest.mark.parametrize("case", MBCONV, ids=lambda c: "%dx%dx%d_c%d_t%d_o%d_s%d" % c)
+def test_fused_inverted_residual_block(case):
+    n, h, w, cin, t, cout, stride = case
+    layers = _mbconv(cin, t, cout, stride, 0)
+    for l in layers:
+        l["src"] = max(l["src"], -1)
+    sess, xd, ref = _mk(layers, "mbconv", n, h, w, cin)
+    last = len(layers) - 1
+    G.check_plan(sess, xd, ref, list(range(last + 1)), [sms()] * (last + 1), "block unfused")
+    for s in (sms(), 5):
+        G.check_plan(sess, xd, ref, [last], [s], "block fused S=%d" % s)
+        assert sess.kernels() == ["mbconv_tc"]
+
+
+def test_two_fused_blocks_in_a_row_and_partial_groups_are_refused():
+    layers = [_conv(8, 24, 1, src=-1)] + _mbconv(24, 6, 24, 1, 1) + _mbconv(24, 6, 32, 2, 4)
+    sess, xd, ref = _mk(layers, "mbconv2", 2, 18, 22, 8)
+    G.check_plan(sess, xd, ref, [0, 3, 6], [sms()] * 3, "two fused blocks")
+    assert sess.kernels() == ["conv_tc", "mbconv_tc", "mbconv_tc"]
+    # depthwise + projection alone is the pattern without an expansion layer (here with a residual)
+    G.check_plan(sess, xd, ref, [0, 1, 3, 6], [sms()] * 4, "expansion alone, then depthwise + projection")
+    assert sess.kernels() == ["conv_tc", "conv_tc", "mbconv_tc", "mbconv_tc"]
+    for ends in ([0, 2, 3, 6], [3, 6]):   # expansion + depthwise alone, or a 1x1 glued in front
+        with pytest.raises(B.DlfError) as e:
+            B.net_set_plan(sess.net, ends, [sms()] * len(ends))
+        assert e.value.status == B.E_PLAN

@@ -122,6 +122,53 @@ def span_is_chain(layers, first, last):
     return True
 
 
+def _pointwise(l):
+    return l["op"] == "conv" and l["groups"] == 1 and l["kh"] == l["kw"] == 1 and l["stride"] == 1 and l["pad"] == 0 and l["pool"] == 0
+
+
+def _depthwise(l):
+    return (l["op"] == "dwconv" and l["kh"] == l["kw"] == 3 and l["pad"] == 1 and l["stride"] in (1, 2) and l["pool"] == 0
+            and l["res_src"] == -2)
+
+
+def span_is_mbconv(layers, first, last, prefix):
+    """Inverted-residual pattern, from its description: [1x1 conv, depthwise 3x3, 1x1 conv] or
+    [depthwise 3x3, 1x1 conv], each reading its predecessor, no pooling, a residual only on the
+    projection and from outside, the maps in between used nowhere else; `prefix` also accepts the
+    pattern's first layers.  Channel limits of the fused kernel: C_in <= 256 (multiple of 8), hidden
+    <= 1024 (multiple of 16), C_out <= 512 (multiple of 8; above 256 a multiple of 32 after padding)."""
+    n_len = last - first + 1
+    if n_len < 2 or n_len > 3:
+        return False
+    has_expand = layers[first]["op"] == "conv"
+    n_full = 3 if has_expand else 2
+    if n_len > n_full or (not prefix and n_len != n_full):
+        return False
+    idx = first
+    if has_expand:
+        if not _pointwise(layers[first]) or layers[first]["res_src"] != -2:
+            return False
+        idx += 1
+    dd = layers[idx]
+    if not _depthwise(dd) or (idx > first and dd["src"] != idx - 1):
+        return False
+    hid, cout = dd["cin"], 8   # no projection yet (a prefix): nothing to check on its width
+    if idx < last:
+        dp = layers[idx + 1]
+        if not _pointwise(dp) or dp["src"] != idx or dp["res_src"] >= first:
+            return False
+        cout = dp["cout"]
+    cin = layers[first]["cin"] if has_expand else hid
+    cpad = (cout + 15) // 16 * 16
+    if cin % 8 or hid % 16 or cout % 8 or cin > 256 or cout > 512 or hid > 1024 or (cpad > 256 and cpad % 32):
+        return False
+    for j in range(first + 1, len(layers)):
+        for which, r in (("src", layers[j]["src"]), ("res", layers[j]["res_src"])):
+            if first <= r < last and not (which == "src" and j <= last and r == j - 1):
+                return False
+    return True
+
+
 P = dict(alpha=0.316, beta=0.659, kappa=12.0, kappa0=-60.0, s_max=148)
 
 
@@ -136,8 +183,18 @@ def test_autotune_equals_restated_algorithm1(name, layers, batch, crit):
     kinds = [l["op"] in ("conv", "dwconv", "fc") for l in layers]
     ch = [l["cout"] for l in layers]
     n = len(layers)
+
+    def can_extend(start, i):   # layers start..i+1 are, or can still become, one fused group
+        return span_is_chain(layers, start, i + 1) or span_is_mbconv(layers, start, i + 1, True)
+
+    def may_close(start, i):    # layers start..i already are a group one kernel runs
+        return i == start or span_is_chain(layers, start, i) or span_is_mbconv(layers, start, i, False)
+
     want = model.algorithm1(kinds, ch, ops, dict(P, op_critical=crit),
-                            must_close_after=lambda start, i: i == n - 1 or not span_is_chain(layers, start, i + 1))
+                            must_close_after=lambda start, i: i == n - 1 or not can_extend(start, i), may_close=may_close)
     got = B.net_autotune(net, n, P["alpha"], P["beta"], P["kappa"], P["kappa0"], crit, s_max=148, legalise=0)
     assert got == (want[0], want[1]), (got, want)
+    if name == "mobilenet_v2" and crit == 1e30:   # every inverted-residual block becomes one group
+        firsts = [0] + [e + 1 for e in got[0][:-1]]
+        assert sum(1 for a, e in zip(firsts, got[0]) if e - a + 1 >= 2) == 17
     B.net_destroy(net)
