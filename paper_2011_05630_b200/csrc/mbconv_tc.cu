@@ -71,7 +71,6 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
     uint8_t* sb = smem_raw + (base - smem_u32(smem_raw));
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &abort_s;
-    float* dw_s = reinterpret_cast<float*>(sb + p.dw_off);      // [9][64] depthwise weights of the chunk, then [64] bias
     float* bias_s = reinterpret_cast<float*>(sb + p.bias_off);  // b1[chunks * 64] then b2[n2_pad]
 
     if (threadIdx.x == 0) {
@@ -225,12 +224,31 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                 if (!ok) break;
             }
             for (int hc = 0; hc < p.chunks && ok; hc++, cc++) {
-                // depthwise weights and bias of the chunk (channels past `hid` are zero)
-                for (int i = wt; i < 640; i += 32 * kWorkWarps) {
-                    const int ch = hc * 64 + (i & 63), tap = i >> 6;
-                    float v = 0.0f;
-                    if (ch < p.hid) v = tap < 9 ? __half2float(__ldg(p.wd + ch * 9 + tap)) : __ldg(p.bd + ch);
-                    dw_s[i] = v;
+                // this thread's depthwise weights and bias: it keeps one 8-channel group of the chunk for all
+                // its pixels (256 threads, 8 groups: the group index is the thread index modulo 8)
+                const int groups = min(8, (p.hid - hc * 64 + 7) >> 3);  // channel groups this chunk really has
+                float wreg[9][8], breg[8];
+                {
+                    const int ch0 = hc * 64 + (wt & 7) * 8;
+                    if ((wt & 7) < groups) {
+                        __align__(16) __half wv[72];
+                        const uint4* wp4 = reinterpret_cast<const uint4*>(p.wd + static_cast<long long>(ch0) * 9);
+#pragma unroll
+                        for (int k = 0; k < 9; k++) reinterpret_cast<uint4*>(wv)[k] = __ldg(wp4 + k);
+#pragma unroll
+                        for (int e = 0; e < 8; e++) {
+                            breg[e] = __ldg(p.bd + ch0 + e);
+#pragma unroll
+                            for (int tp = 0; tp < 9; tp++) wreg[tp][e] = __half2float(wv[e * 9 + tp]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 8; e++) {
+                            breg[e] = 0.0f;
+#pragma unroll
+                            for (int tp = 0; tp < 9; tp++) wreg[tp][e] = 0.0f;
+                        }
+                    }
                 }
                 if (p.has_expand) {
                     // ---- epilogue 1: D1 -> H (fp16, zero outside the image) ------------------------------
@@ -265,7 +283,7 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&d1_free);
                 }
-                work_bar_sync();  // H (and the depthwise weights) complete
+                work_bar_sync();  // H complete
                 if (cc > 0) {
                     ok = mbar_wait(&hd_free, (cc - 1) & 1u, abort_flag, p.status, 0xE20 | (blockIdx.x << 12));
                     if (!ok) break;
@@ -274,38 +292,42 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                 const uint8_t* hsrc = hbuf + (p.has_expand ? 0 : hc * p.nb1 * kPlane);
                 for (int item = wt; item < p.th * p.tw * 8; item += 32 * kWorkWarps) {
                     const int g8 = item & 7, o = item >> 3;
-                    const int oy = o / p.tw, ox = o - oy * p.tw;
-                    float acc[8];
+                    uint4 val = make_uint4(0u, 0u, 0u, 0u);  // groups the chunk does not have: zero operand columns
+                    if (g8 < groups) {
+                        const int oy = o / p.tw, ox = o - oy * p.tw;
+                        float acc[8];
 #pragma unroll
-                    for (int e = 0; e < 8; e++) acc[e] = 0.0f;
+                        for (int e = 0; e < 8; e++) acc[e] = 0.0f;
+                        uint4 xv[9];
 #pragma unroll
-                    for (int r = 0; r < 3; r++)
+                        for (int r = 0; r < 3; r++)
 #pragma unroll
-                        for (int c = 0; c < 3; c++) {
-                            const int qrow = (oy * p.stride + r) * p.fw + ox * p.stride + c;
-                            const uint4 xv = *reinterpret_cast<const uint4*>(hsrc + qrow * 128 + ((g8 ^ (qrow & 7)) << 4));
-                            const __half2* xh = reinterpret_cast<const __half2*>(&xv);
-                            const float* wv = dw_s + (r * 3 + c) * 64 + g8 * 8;
+                            for (int c = 0; c < 3; c++) {
+                                const int qrow = (oy * p.stride + r) * p.fw + ox * p.stride + c;
+                                xv[r * 3 + c] = *reinterpret_cast<const uint4*>(hsrc + qrow * 128 + ((g8 ^ (qrow & 7)) << 4));
+                            }
+#pragma unroll
+                        for (int tp = 0; tp < 9; tp++) {
+                            const __half2* xh = reinterpret_cast<const __half2*>(&xv[tp]);
 #pragma unroll
                             for (int e = 0; e < 4; e++) {
                                 const float2 f = __half22float2(xh[e]);
-                                acc[2 * e] = fmaf(f.x, wv[2 * e], acc[2 * e]);
-                                acc[2 * e + 1] = fmaf(f.y, wv[2 * e + 1], acc[2 * e + 1]);
+                                acc[2 * e] = fmaf(f.x, wreg[tp][2 * e], acc[2 * e]);
+                                acc[2 * e + 1] = fmaf(f.y, wreg[tp][2 * e + 1], acc[2 * e + 1]);
                             }
                         }
-                    const float* bv = dw_s + 576 + g8 * 8;
-                    uint4 val;
-                    val.x = pack_half2(clampf(acc[0] + bv[0], lo2, hi2), clampf(acc[1] + bv[1], lo2, hi2));
-                    val.y = pack_half2(clampf(acc[2] + bv[2], lo2, hi2), clampf(acc[3] + bv[3], lo2, hi2));
-                    val.z = pack_half2(clampf(acc[4] + bv[4], lo2, hi2), clampf(acc[5] + bv[5], lo2, hi2));
-                    val.w = pack_half2(clampf(acc[6] + bv[6], lo2, hi2), clampf(acc[7] + bv[7], lo2, hi2));
+                        val.x = pack_half2(clampf(acc[0] + breg[0], lo2, hi2), clampf(acc[1] + breg[1], lo2, hi2));
+                        val.y = pack_half2(clampf(acc[2] + breg[2], lo2, hi2), clampf(acc[3] + breg[3], lo2, hi2));
+                        val.z = pack_half2(clampf(acc[4] + breg[4], lo2, hi2), clampf(acc[5] + breg[5], lo2, hi2));
+                        val.w = pack_half2(clampf(acc[6] + breg[6], lo2, hi2), clampf(acc[7] + breg[7], lo2, hi2));
+                    }
                     *reinterpret_cast<uint4*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4)) = val;
                 }
                 fence_proxy_async_smem();  // the projection UMMAs read Hd through the async proxy
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&hd_ready);
                 if (!p.has_expand && hc + 1 == p.chunks && lane == 0) mbar_arrive(&x_empty);
-                work_bar_sync();  // nobody still reads H / the depthwise weights when the next chunk overwrites them
+                work_bar_sync();  // nobody still reads H when the next chunk overwrites it
             }
             if (!ok) break;
             // ---- epilogue 2: D2 -> global -------------------------------------------------------------------
@@ -407,7 +429,7 @@ MbconvTiling mbconv_tiling(const MbconvArgs& a, int sm_count) {
             if (n_tiles > 0x7fffffffLL) continue;
             const long long waves = (n_tiles + sm_count - 1) / sm_count;
             // per chunk: epilogue-1 rows + depthwise items on 256 threads, plus hand-off latency
-            const double per_chunk = (a.has_expand ? nb1 * 128 * 2.0 : 0.0) + th * tw * 8 * 6.0 + 1500.0;
+            const double per_chunk = (a.has_expand ? nb1 * 128 * 1.5 : 0.0) + th * tw * 4.0 + 2500.0;
             const double cost = static_cast<double>(waves) * (chunks * per_chunk + 3000.0);
             if (best_cost < 0 || cost < best_cost) {
                 best_cost = cost;
