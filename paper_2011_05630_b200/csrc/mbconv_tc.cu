@@ -61,6 +61,54 @@ __device__ __forceinline__ void work_bar_sync() { asm volatile("bar.sync 1, %0;"
 
 __device__ __forceinline__ float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi); }
 
+// Depthwise 3x3 of one 8-channel group for two horizontally adjacent output pixels: the input
+// vectors the two windows share are read from shared memory and converted once.
+template <int STRIDE>
+__device__ __forceinline__ void dw_pair(const uint8_t* hsrc, uint8_t* hdbuf, int fw, int tw, int g8, int oy, int ox, bool second,
+                                        const float (&wreg)[9][8], const float (&breg)[8], float lo, float hi) {
+    constexpr int kCols = STRIDE + 3;  // input columns the two windows cover
+    float acc[2][8];
+#pragma unroll
+    for (int e = 0; e < 8; e++) acc[0][e] = acc[1][e] = 0.0f;
+#pragma unroll
+    for (int r = 0; r < 3; r++) {
+        const int q0 = (oy * STRIDE + r) * fw + ox * STRIDE;
+        uint4 xv[kCols];
+#pragma unroll
+        for (int c = 0; c < kCols; c++) xv[c] = *reinterpret_cast<const uint4*>(hsrc + (q0 + c) * 128 + ((g8 ^ ((q0 + c) & 7)) << 4));
+#pragma unroll
+        for (int c = 0; c < kCols; c++) {
+            const __half2* xh = reinterpret_cast<const __half2*>(&xv[c]);
+            float xf[8];
+#pragma unroll
+            for (int e = 0; e < 4; e++) {
+                const float2 f = __half22float2(xh[e]);
+                xf[2 * e] = f.x;
+                xf[2 * e + 1] = f.y;
+            }
+            if (c < 3) {
+#pragma unroll
+                for (int e = 0; e < 8; e++) acc[0][e] = fmaf(xf[e], wreg[r * 3 + c][e], acc[0][e]);
+            }
+            if (c >= STRIDE) {
+#pragma unroll
+                for (int e = 0; e < 8; e++) acc[1][e] = fmaf(xf[e], wreg[r * 3 + c - STRIDE][e], acc[1][e]);
+            }
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < 2; k++) {
+        if (k == 1 && !second) break;
+        const int o = oy * tw + ox + k;
+        uint4 val;
+        val.x = pack_half2(clampf(acc[k][0] + breg[0], lo, hi), clampf(acc[k][1] + breg[1], lo, hi));
+        val.y = pack_half2(clampf(acc[k][2] + breg[2], lo, hi), clampf(acc[k][3] + breg[3], lo, hi));
+        val.z = pack_half2(clampf(acc[k][4] + breg[4], lo, hi), clampf(acc[k][5] + breg[5], lo, hi));
+        val.w = pack_half2(clampf(acc[k][6] + breg[6], lo, hi), clampf(acc[k][7] + breg[7], lo, hi));
+        *reinterpret_cast<uint4*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4)) = val;
+    }
+}
+
 __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_constant__ MbParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t x_full, x_empty, w_full[4], w_empty[4], d1_full, d1_free, hd_ready, hd_free, d2_full, d2_free;
@@ -269,10 +317,11 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                             for (int g = 0; g < 4; g++) {
                                 uint4 val = make_uint4(0u, 0u, 0u, 0u);
                                 if (in_img) {
-                                    val.x = pack_half2(clampf(v[g * 8 + 0] + bb[g * 8 + 0], lo1, hi1), clampf(v[g * 8 + 1] + bb[g * 8 + 1], lo1, hi1));
-                                    val.y = pack_half2(clampf(v[g * 8 + 2] + bb[g * 8 + 2], lo1, hi1), clampf(v[g * 8 + 3] + bb[g * 8 + 3], lo1, hi1));
-                                    val.z = pack_half2(clampf(v[g * 8 + 4] + bb[g * 8 + 4], lo1, hi1), clampf(v[g * 8 + 5] + bb[g * 8 + 5], lo1, hi1));
-                                    val.w = pack_half2(clampf(v[g * 8 + 6] + bb[g * 8 + 6], lo1, hi1), clampf(v[g * 8 + 7] + bb[g * 8 + 7], lo1, hi1));
+                                    const float4 ba = *reinterpret_cast<const float4*>(bb + g * 8), bc = *reinterpret_cast<const float4*>(bb + g * 8 + 4);
+                                    val.x = pack_half2(clampf(v[g * 8 + 0] + ba.x, lo1, hi1), clampf(v[g * 8 + 1] + ba.y, lo1, hi1));
+                                    val.y = pack_half2(clampf(v[g * 8 + 2] + ba.z, lo1, hi1), clampf(v[g * 8 + 3] + ba.w, lo1, hi1));
+                                    val.z = pack_half2(clampf(v[g * 8 + 4] + bc.x, lo1, hi1), clampf(v[g * 8 + 5] + bc.y, lo1, hi1));
+                                    val.w = pack_half2(clampf(v[g * 8 + 6] + bc.z, lo1, hi1), clampf(v[g * 8 + 7] + bc.w, lo1, hi1));
                                 }
                                 const int g8 = half * 4 + g;
                                 *reinterpret_cast<uint4*>(hbuf + r * 128 + ((g8 ^ (r & 7)) << 4)) = val;
@@ -290,38 +339,21 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                 }
                 // ---- depthwise 3x3: H -> Hd ---------------------------------------------------------------
                 const uint8_t* hsrc = hbuf + (p.has_expand ? 0 : hc * p.nb1 * kPlane);
-                for (int item = wt; item < p.th * p.tw * 8; item += 32 * kWorkWarps) {
-                    const int g8 = item & 7, o = item >> 3;
-                    uint4 val = make_uint4(0u, 0u, 0u, 0u);  // groups the chunk does not have: zero operand columns
+                const int pairs_w = (p.tw + 1) >> 1;
+                for (int item = wt; item < p.th * pairs_w * 8; item += 32 * kWorkWarps) {
+                    const int g8 = item & 7, pr = item >> 3;
+                    const int oy = pr / pairs_w, ox = (pr - oy * pairs_w) * 2;
+                    const bool second = ox + 1 < p.tw;
                     if (g8 < groups) {
-                        const int oy = o / p.tw, ox = o - oy * p.tw;
-                        float acc[8];
-#pragma unroll
-                        for (int e = 0; e < 8; e++) acc[e] = 0.0f;
-                        uint4 xv[9];
-#pragma unroll
-                        for (int r = 0; r < 3; r++)
-#pragma unroll
-                            for (int c = 0; c < 3; c++) {
-                                const int qrow = (oy * p.stride + r) * p.fw + ox * p.stride + c;
-                                xv[r * 3 + c] = *reinterpret_cast<const uint4*>(hsrc + qrow * 128 + ((g8 ^ (qrow & 7)) << 4));
-                            }
-#pragma unroll
-                        for (int tp = 0; tp < 9; tp++) {
-                            const __half2* xh = reinterpret_cast<const __half2*>(&xv[tp]);
-#pragma unroll
-                            for (int e = 0; e < 4; e++) {
-                                const float2 f = __half22float2(xh[e]);
-                                acc[2 * e] = fmaf(f.x, wreg[tp][2 * e], acc[2 * e]);
-                                acc[2 * e + 1] = fmaf(f.y, wreg[tp][2 * e + 1], acc[2 * e + 1]);
-                            }
-                        }
-                        val.x = pack_half2(clampf(acc[0] + breg[0], lo2, hi2), clampf(acc[1] + breg[1], lo2, hi2));
-                        val.y = pack_half2(clampf(acc[2] + breg[2], lo2, hi2), clampf(acc[3] + breg[3], lo2, hi2));
-                        val.z = pack_half2(clampf(acc[4] + breg[4], lo2, hi2), clampf(acc[5] + breg[5], lo2, hi2));
-                        val.w = pack_half2(clampf(acc[6] + breg[6], lo2, hi2), clampf(acc[7] + breg[7], lo2, hi2));
+                        // the second window of a last, odd pair reads columns past the frame row: still inside the
+                        // buffer (next row or slack), and its result is not stored
+                        if (p.stride == 1) dw_pair<1>(hsrc, hdbuf, p.fw, p.tw, g8, oy, ox, second, wreg, breg, lo2, hi2);
+                        else dw_pair<2>(hsrc, hdbuf, p.fw, p.tw, g8, oy, ox, second, wreg, breg, lo2, hi2);
+                    } else {  // channel groups the chunk does not have: zero operand columns
+                        const int o = oy * p.tw + ox;
+                        *reinterpret_cast<uint4*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                        if (second) *reinterpret_cast<uint4*>(hdbuf + (o + 1) * 128 + ((g8 ^ ((o + 1) & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
                     }
-                    *reinterpret_cast<uint4*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4)) = val;
                 }
                 fence_proxy_async_smem();  // the projection UMMAs read Hd through the async proxy
                 __syncwarp();

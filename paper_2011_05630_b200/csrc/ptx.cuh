@@ -70,6 +70,8 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     uint32_t spins = 0;
     while (true) {
         if (mbar_try_wait(bar, parity)) return true;
+        // back off: a spinning single-thread role shares its scheduler with the warps doing the work
+        if (spins > 4) __nanosleep(spins > 64 ? 128 : 32);
         if ((++spins & 63u) == 0) {
             if (*abort_flag) return false;
             if (global_ns() - t0 > kWaitLimitNs) {
