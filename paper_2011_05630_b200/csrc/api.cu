@@ -181,7 +181,12 @@ static bool depthwise_ok(const dlf_layer_desc& d) {
     return d.op == DLF_DWCONV && d.kh == 3 && d.kw == 3 && d.pad == 1 && (d.stride == 1 || d.stride == 2) && d.pool == 0 &&
            d.res_src == -2;
 }
-static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix) {
+// Widest hidden tensor of an inverted-residual block the tuner proposes as one kernel: the kernel walks
+// the hidden channels in 64-wide steps one after the other, and beyond four steps three kernels that
+// each fill the chip were measured faster.  A plan given explicitly may still ask for a wider block.
+static const int kTunerMaxHidden = 256;
+
+static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix, int max_hid = 0) {
     const int len = last - first + 1;
     if (len < 2 || len > 3) return false;
     const dlf_layer_desc& d0 = net->layers[first].d;
@@ -205,7 +210,7 @@ static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix)
     std::memset(&a, 0, sizeof(a));
     a.N = 1; a.H = 8; a.W = 8;
     a.Cin = has_expand ? d0.cin : hid; a.hid = hid; a.Cout = cout; a.stride = dd.stride; a.has_expand = has_expand ? 1 : 0;
-    if (!mbconv_supported(a)) return false;
+    if (!mbconv_supported(a) || (max_hid > 0 && hid > max_hid)) return false;
     // the maps between the layers are used nowhere else
     const int n = static_cast<int>(net->layers.size());
     for (int j = first + 1; j < n; j++) {
@@ -726,11 +731,11 @@ int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_
         }
         // a block may grow while its layers are, or can still become, a group one kernel runs; it may
         // close only where they already are one (inside an inverted-residual block it keeps growing)
-        bool forced = (i == n - 1) || !(span_is_chain(net, start, i + 1) || span_is_mbconv(net, start, i + 1, true));
-        const bool closable = (i == start) || span_is_chain(net, start, i) || span_is_mbconv(net, start, i, false);
+        bool forced = (i == n - 1) || !(span_is_chain(net, start, i + 1) || span_is_mbconv(net, start, i + 1, true, kTunerMaxHidden));
+        const bool closable = (i == start) || span_is_chain(net, start, i) || span_is_mbconv(net, start, i, false, kTunerMaxHidden);
         if (!forced && params->legalise) {
             Group g;
-            if (i + 1 > start && (span_is_chain(net, start, i + 1) || span_is_mbconv(net, start, i + 1, false)))
+            if (i + 1 > start && (span_is_chain(net, start, i + 1) || span_is_mbconv(net, start, i + 1, false, kTunerMaxHidden)))
                 forced = !make_group(net, start, i + 1, s_max, &g);
         }
         if (block > 0) {

@@ -34,9 +34,18 @@ def test_network_every_boundary(name, builder, batch):
     todo = [("unfused", None, None)]
     ends, smc = plans.tuned_plan(sess.net, len(layers))
     todo.append(("tuned", ends, smc))
-    if name == "mobilenet_v2":   # one group per inverted-residual block (the critical op count set out of reach)
-        ends, smc = plans.tuned_plan(sess.net, len(layers), op_critical=1e30)
-        todo.append(("block-fused", ends, smc))
+    if name == "mobilenet_v2":   # every inverted-residual block as one group, the wide ones the tuner leaves apart too
+        ends, i = [], 0
+        while i < len(layers):
+            span = 1
+            if layers[i]["op"] == "dwconv" or (i + 1 < len(layers) and layers[i + 1]["op"] == "dwconv"):
+                span = 2 if layers[i]["op"] == "dwconv" else 3
+                if B.net_group_is_legal(sess.net, i, i + span - 1, sms) != 1:
+                    span = 1
+            ends.append(i + span - 1)
+            i += span
+        assert sum(1 for a, e in zip([0] + [e + 1 for e in ends[:-1]], ends) if e > a) == 17
+        todo.append(("block-fused", ends, [sms] * len(ends)))
     for what, e, s in todo:
         ends_now, _ = sess.set_plan(e, s)
         out = sess.run(xd).cpu().numpy()
