@@ -23,8 +23,15 @@ __device__ __forceinline__ uint64_t global_ns() {
 // a few points after the status word.
 #ifdef DLF_TRACE
 #define DLF_TRACE_POINT(status, slot) do { if (blockIdx.x == 0) reinterpret_cast<volatile unsigned long long*>(status)[4 + (slot)] = global_ns(); } while (0)
+// per-phase cycle sums of CTA 0's thread 0: ACC adds the cycles since the last mark to a slot
+#define DLF_TRACE_DECL(acc, mark) long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long mark = clock64()
+#define DLF_TRACE_ACC(acc, slot, mark) do { const long long now_ = clock64(); acc[slot] += now_ - mark; mark = now_; } while (0)
+#define DLF_TRACE_FLUSH(status, acc) do { if (blockIdx.x == 0 && threadIdx.x == 0) for (int i_ = 0; i_ < 8; i_++) reinterpret_cast<volatile long long*>(status)[4 + i_] = acc[i_]; } while (0)
 #else
 #define DLF_TRACE_POINT(status, slot) do { } while (0)
+#define DLF_TRACE_DECL(acc, mark) do { } while (0)
+#define DLF_TRACE_ACC(acc, slot, mark) do { } while (0)
+#define DLF_TRACE_FLUSH(status, acc) do { } while (0)
 #endif
 
 // ---- programmatic dependent launch -----------------------------------------------------------------
@@ -195,6 +202,8 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* m, const void* s
 __device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 // Waits until the committed stores have finished READING shared memory (the buffer may be reused).
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... all but the newest committed store have finished reading.
+__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // The barrier gets one arrival when every UMMA issued so far by this thread has completed.

@@ -66,6 +66,9 @@ SINGLE = [
     (9, 7, 7, _conv(512, 512, 3)),                 # several images per tile
     (2, 33, 35, _conv(3, 32, 3, stride=2, act="relu6")),   # C = 3 stem (direct kernel)
     (1, 45, 43, _conv(3, 64, 7, stride=2, pad=3)),
+    (2, 37, 29, _conv(3, 64, 3)),                          # stride 1: patch rows start on odd halves
+    (3, 30, 31, _conv(4, 16, 5, stride=2, pad=2, act="none")),
+    (5, 6, 6, _conv(3, 24, 3, stride=2)),                  # several images per tile
     (2, 20, 20, _conv(3, 64, 3, pool=2)),
     (2, 21, 22, _conv(96, 96, 3, stride=1, act="relu6", groups=96, op="dwconv")),
     (2, 21, 22, _conv(144, 144, 3, stride=2, act="relu6", groups=144, op="dwconv")),
