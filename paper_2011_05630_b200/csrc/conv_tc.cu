@@ -13,8 +13,13 @@
 // tcgen05.mma (fp16 x fp16 -> fp32) into one of two TMEM accumulators; eight epilogue warps (two
 // per TMEM lane quarter, alternating 32-column chunks) drain the other accumulator: bias (staged
 // in shared memory), residual, activation, fp16 rounding.  Without pooling the tile is written to
-// a swizzled staging buffer and leaves through TMA stores (clipped at the tensor's edges); with
-// the fused 2x2 max-pool the window is reduced by warp shuffles and written with 16-byte stores.
+// a swizzled staging buffer (two of them where the ring leaves room) and a separate warp sends it
+// off with TMA stores (clipped at the tensor's edges), waits until they have read the buffer and hands
+// it back - so the epilogue warps never wait for a store.  A residual is fetched by that same warp
+// with TMA loads straight INTO the staging buffer one or two tiles ahead and added in place: with one
+// output pixel per thread, direct residual loads would touch 32 cache lines per instruction and
+// were measured to double the time of the memory-bound 1x1 layers.  With the fused 2x2 max-pool
+// the window is reduced by warp shuffles and written with 16-byte stores.
 // The epilogue is specialised at compile time on (activation, pool, residual): it is the part of
 // the kernel that bounds memory-bound layers, and runtime branches there cost more than the math.
 #include <cuda.h>
@@ -32,7 +37,8 @@ namespace {
 constexpr int kEpiWarps = 8;
 constexpr int kMmaWarp = kEpiWarps;         // warps 0..7 epilogue (warp & 3 = TMEM lane quarter), 8 UMMA issuer,
 constexpr int kProdWarp0 = kEpiWarps + 1;   // 9..12 producers: A even / A odd / B even / B odd ring stages
-constexpr int kThreads = 32 * (kEpiWarps + 5);
+constexpr int kStoreWarp = kProdWarp0 + 4;  // 13: TMA stores of finished tiles, TMA loads of residual tiles
+constexpr int kThreads = 32 * (kEpiWarps + 6);
 constexpr int kABytes = 128 * 128;  // 128 pixels x 64 fp16
 constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
 
@@ -46,6 +52,7 @@ struct ConvTcParams {
     int stages;
     int n_work;
     int stage_out_off, bias_off;  // byte offsets in dynamic shared memory
+    int out_bufs, out_buf_bytes;  // staging buffers (1 or 2) and the size of one
     uint32_t tmem_cols;
     const float* bias;
     const __half* res;
@@ -69,14 +76,13 @@ __device__ __forceinline__ TileCoord decode_work(const ConvTcParams& p, int t) {
     return c;
 }
 
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory"); }
-
 template <int ACT, bool POOL, bool RES>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
-               const __grid_constant__ CUtensorMap tmy, const ConvTcParams p) {
+               const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmr, const ConvTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[8], empty_bar[8], tfull_bar[2], tempty_bar[2];
+    __shared__ uint64_t sfull_bar[2], sfree_bar[2];  // staging buffer: filled by the epilogue / free again (residual landed)
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
@@ -97,11 +103,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         for (int i = 0; i < 2; i++) {
             mbar_init(&tfull_bar[i], 1);
             mbar_init(&tempty_bar[i], kEpiWarps);
+            mbar_init(&sfull_bar[i], kEpiWarps);
+            mbar_init(&sfree_bar[i], 1);
         }
         fence_barrier_init();
         tma_prefetch_desc(&tmx);
         tma_prefetch_desc(&tmw);
         if (!POOL) tma_prefetch_desc(&tmy);
+        if (!POOL && RES) tma_prefetch_desc(&tmr);
     }
     if (warp == kMmaWarp) {
         tmem_alloc(&tmem_base_s, p.tmem_cols);
@@ -117,13 +126,46 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     pdl_launch_dependents();
     // everything above overlapped the previous kernel; from here on its outputs are read - except by the
     // weight producers, which only read constants and may run ahead
-    if (warp < kProdWarp0 + 2) pdl_wait();
+    if (warp < kProdWarp0 + 2 || warp == kStoreWarp) pdl_wait();
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
     const int taps = p.kh * p.kw;
     const int k_iters = taps * p.kgroups;
 
-    if (warp >= kProdWarp0) {
+    if (warp == kStoreWarp) {
+        // ---- staging buffers out (TMA stores) and residual tiles in (TMA loads) ------------------------
+        if (!POOL && lane == 0) {
+            uint8_t* stage_out = stage0 + p.stage_out_off;
+            auto planes_of = [&](const TileCoord& c) { return (min(p.BN, ((p.Cout - c.co0) + 15) & ~15) + 63) >> 6; };
+            auto fetch_residual = [&](int t, uint32_t b) {
+                const TileCoord c = decode_work(p, t);
+                const int planes = planes_of(c);
+                mbar_expect_tx(&sfree_bar[b], static_cast<uint32_t>(planes) * kABytes);
+                for (int pl = 0; pl < planes; pl++)
+                    tma_load_4d(stage_out + b * p.out_buf_bytes + pl * kABytes, &tmr, &sfree_bar[b], c.co0 + pl * 64, c.wo0, c.ho0, c.n0);
+            };
+            if (RES)
+                for (int jj = 0; jj < p.out_bufs; jj++)
+                    if (static_cast<int>(blockIdx.x) + jj * static_cast<int>(gridDim.x) < p.n_work) fetch_residual(blockIdx.x + jj * gridDim.x, jj);
+            uint32_t j = 0;
+            for (int t = blockIdx.x; t < p.n_work; t += gridDim.x, j++) {
+                const uint32_t b = j % p.out_bufs, ph = (j / p.out_bufs) & 1u;
+                if (!mbar_wait(&sfull_bar[b], ph, abort_flag, p.status, 0x500 | (blockIdx.x << 12))) break;
+                const TileCoord c = decode_work(p, t);
+                const int planes = planes_of(c);
+                for (int pl = 0; pl < planes; pl++)
+                    tma_store_4d(&tmy, stage_out + b * p.out_buf_bytes + pl * kABytes, c.co0 + pl * 64, c.wo0, c.ho0, c.n0);
+                tma_store_commit();
+                tma_store_wait_read();  // the buffer has been read: it may take the next residual / the next tile
+                const int t2 = t + p.out_bufs * static_cast<int>(gridDim.x);
+                if (RES) {
+                    if (t2 < p.n_work) fetch_residual(t2, b);
+                } else {
+                    mbar_arrive(&sfree_bar[b]);
+                }
+            }
+        }
+    } else if (warp >= kProdWarp0) {
         // ---- producers: TMA loads into the stage ring -------------------------------------------
         if (lane == 0) {
             const int role = warp - kProdWarp0;
@@ -210,21 +252,44 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
             const TileCoord c = decode_work(p, t);
             const uint32_t acc = j & 1u;
-            ok = mbar_wait(&tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
-            if (!ok) break;
-            if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 5);
-            tc_fence_after_sync();
             const int n = c.n0 + tn, ho = c.ho0 + th, wo = c.wo0 + tw;
             const bool valid = n < p.N && ho < p.Ho && wo < p.Wo;
             const long long pix = (static_cast<long long>(n) * p.Ho + ho) * p.Wo + wo;
             const long long opix = POOL ? (static_cast<long long>(n) * Hp + (ho >> 1)) * Wp + (wo >> 1) : pix;
             const bool writer = valid && (!POOL || (((ho | wo) & 1) == 0 && (ho >> 1) < Hp && (wo >> 1) < Wp));
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.acc_stride;
             const int ncols = min(p.BN, ((p.Cout - c.co0) + 15) & ~15);
+            // The residual of this pixel's next 32 channels, four 16-byte loads issued together without a
+            // branch (clamped address; `rok` keeps which are real): fetched one column pass ahead, the first
+            // before the accumulator is even complete, so that their latency is never waited for.
+            uint4 rcur[4], rnext[4];
+            uint32_t rok = 0u, rok_next = 0u;
+            auto res_load = [&](int cc, uint4 (&rv)[4], uint32_t& okm) {
+                okm = 0u;
+#pragma unroll
+                for (int g = 0; g < 4; g++) {
+                    const int co = c.co0 + cc + g * 8;
+                    const bool okg = valid && cc + g * 8 < ncols && co < p.Cout;
+                    rv[g] = __ldg(reinterpret_cast<const uint4*>(p.res + (okg ? pix * p.Cout + co : 0)));
+                    okm |= (okg ? 1u : 0u) << g;
+                }
+            };
+            if (RES && POOL) res_load(half * 32, rcur, rok);
+            uint8_t* sout = stage_out + (j % p.out_bufs) * p.out_buf_bytes;
+            if (!POOL) {   // the staging buffer is free (first uses pass at once) / holds this tile's residual
+                const uint32_t ph = (j / p.out_bufs) & 1u;
+                ok = mbar_wait(&sfree_bar[j % p.out_bufs], RES ? ph : ph ^ 1u, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
+                if (!ok) break;
+            }
+            ok = mbar_wait(&tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
+            if (!ok) break;
+            if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 5);
+            tc_fence_after_sync();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.acc_stride;
             for (int cc = half * 32; cc < ncols; cc += 64) {
                 float v[32];
                 __syncwarp();  // the aligned TMEM load needs the whole warp converged
                 const int nc = min(32, ncols - cc);
+                if (RES && POOL && cc + 64 < ncols) res_load(cc + 64, rnext, rok_next);
                 if (nc == 32) tmem_ld32(taddr + cc, v);
                 else tmem_ld16(taddr + cc, v);
 #pragma unroll
@@ -236,16 +301,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     const float4 b1 = *reinterpret_cast<const float4*>(bias_s + co + 4);
                     a[0] = v[g * 8 + 0] + b0.x; a[1] = v[g * 8 + 1] + b0.y; a[2] = v[g * 8 + 2] + b0.z; a[3] = v[g * 8 + 3] + b0.w;
                     a[4] = v[g * 8 + 4] + b1.x; a[5] = v[g * 8 + 5] + b1.y; a[6] = v[g * 8 + 6] + b1.z; a[7] = v[g * 8 + 7] + b1.w;
-                    if (RES) {
-                        if (valid && co < p.Cout) {
-                            const uint4 rv = __ldg(reinterpret_cast<const uint4*>(p.res + pix * p.Cout + co));
-                            const __half2* rh = reinterpret_cast<const __half2*>(&rv);
+                    const int g8 = (cc >> 3) + g;
+                    uint4* sptr = reinterpret_cast<uint4*>(sout + (g8 >> 3) * kABytes + m * 128 + (((g8 & 7) ^ (m & 7)) << 4));
+                    if (RES && !POOL) {   // the residual tile was loaded into the staging buffer (zero outside the tensor)
+                        const uint4 rv = *sptr;
+                        const __half2* rh = reinterpret_cast<const __half2*>(&rv);
 #pragma unroll
-                            for (int e = 0; e < 4; e++) {
-                                const float2 f = __half22float2(rh[e]);
-                                a[2 * e] += f.x;
-                                a[2 * e + 1] += f.y;
-                            }
+                        for (int e = 0; e < 4; e++) {
+                            const float2 f = __half22float2(rh[e]);
+                            a[2 * e] += f.x;
+                            a[2 * e + 1] += f.y;
+                        }
+                    }
+                    if (RES && POOL) {
+                        const bool okg = (rok >> g) & 1u;
+                        const __half2* rh = reinterpret_cast<const __half2*>(&rcur[g]);
+#pragma unroll
+                        for (int e = 0; e < 4; e++) {
+                            const float2 f = __half22float2(rh[e]);
+                            a[2 * e] += okg ? f.x : 0.0f;
+                            a[2 * e + 1] += okg ? f.y : 0.0f;
                         }
                     }
                     uint4 o;
@@ -262,9 +337,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     if (POOL) {
                         if (writer && co < p.Cout) *reinterpret_cast<uint4*>(p.out + opix * p.Cout + co) = o;
                     } else {
-                        const int g8 = (cc >> 3) + g;
-                        *reinterpret_cast<uint4*>(stage_out + (g8 >> 3) * kABytes + m * 128 + (((g8 & 7) ^ (m & 7)) << 4)) = o;
+                        *sptr = o;
                     }
+                }
+                if (RES && POOL) {
+#pragma unroll
+                    for (int g = 0; g < 4; g++) rcur[g] = rnext[g];
+                    rok = rok_next;
                 }
             }
             tc_fence_before_sync();
@@ -272,18 +351,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             if (lane == 0) mbar_arrive(&tempty_bar[acc]);  // the accumulator is drained
             if (!POOL) {
                 fence_proxy_async_smem();  // the staging tile is read by the TMA unit
-                epi_bar_sync();
-                if (lane == 0 && warp * 64 < ncols) {  // one 64-channel plane per warp: TMA issue is slow per thread
-                    tma_store_4d(&tmy, stage_out + warp * kABytes, c.co0 + warp * 64, c.wo0, c.ho0, c.n0);
-                    tma_store_commit();
-                    tma_store_wait_read();
-                }
-                epi_bar_sync();  // the staging tile may be overwritten
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sfull_bar[j % p.out_bufs]);
             }
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 6);
         }
-        if (!POOL && lane == 0) tma_store_wait_read();  // the staging tile must outlive the stores' reads; the grid's
-                                                        // completion makes their writes visible
     }
 
     tc_fence_before_sync();
@@ -318,7 +390,7 @@ Tile pick_tile(int N, int Ho, int Wo, int pool) {
     return best;
 }
 
-typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const ConvTcParams);
+typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const ConvTcParams);
 
 template <int ACT, bool POOL>
 KernelFn pick_res(bool res) {
@@ -384,23 +456,30 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     p.ksteps_last = ((a.Cin - (p.kchunks - 1) * 64) + 15) / 16;
     const int out_planes = a.pool ? 0 : (p.BN + 63) / 64;
     const int bias_bytes = (p.n_tiles_n * p.BN * 4 + 1023) / 1024 * 1024;
-    const int fixed = out_planes * kABytes + bias_bytes + 1024;
-    // K chunks per ring stage: every stage costs the issuing threads a fixed handshake (barrier wait,
-    // TMA issue, commit), so a stage carries as many 64-channel chunks as leave room for >= 2 stages
     p.grouped = (a.Cin % 64 == 0) ? 1 : 0;
-    p.kg = 1;
-    if (p.grouped)
-        for (int kg : {4, 2})
-            if (kg <= p.kchunks && 2 * kg * (kABytes + p.BN * 128) <= kMaxSmem - fixed && (kg == 2 || 3 * kg * (kABytes + p.BN * 128) <= kMaxSmem - fixed || a.kh * a.kw * ((p.kchunks + kg - 1) / kg) <= 2)) {
-                p.kg = kg;
-                break;
-            }
-    p.kgroups = (p.kchunks + p.kg - 1) / p.kg;
-    const int stage_bytes = p.kg * (kABytes + p.BN * 128);
-    p.stages = std::min(6, (kMaxSmem - fixed) / stage_bytes);
-    p.stages = std::max(1, std::min(p.stages, a.kh * a.kw * p.kgroups));
-    p.stage_out_off = p.stages * stage_bytes;
-    p.bias_off = p.stage_out_off + out_planes * kABytes;
+    p.out_buf_bytes = out_planes * kABytes;
+    // Two staging buffers (the stores of one tile drain while the next is written) where the ring keeps
+    // three stages, or as many as the tile has loads, beside them; else one.
+    for (p.out_bufs = a.pool ? 1 : 2; p.out_bufs >= 1; p.out_bufs--) {
+        const int fixed = p.out_bufs * p.out_buf_bytes + bias_bytes + 1024;
+        // K chunks per ring stage: every stage costs the issuing threads a fixed handshake (barrier wait,
+        // TMA issue, commit), so a stage carries as many 64-channel chunks as leave room for >= 2 stages
+        p.kg = 1;
+        if (p.grouped)
+            for (int kg : {4, 2})
+                if (kg <= p.kchunks && 2 * kg * (kABytes + p.BN * 128) <= kMaxSmem - fixed && (kg == 2 || 3 * kg * (kABytes + p.BN * 128) <= kMaxSmem - fixed || a.kh * a.kw * ((p.kchunks + kg - 1) / kg) <= 2)) {
+                    p.kg = kg;
+                    break;
+                }
+        p.kgroups = (p.kchunks + p.kg - 1) / p.kg;
+        const int stage_bytes = p.kg * (kABytes + p.BN * 128);
+        p.stages = std::min(6, (kMaxSmem - fixed) / stage_bytes);
+        const int loads = a.kh * a.kw * p.kgroups;
+        p.stages = std::max(1, std::min(p.stages, loads));
+        p.stage_out_off = p.stages * stage_bytes;
+        p.bias_off = p.stage_out_off + p.out_bufs * p.out_buf_bytes;
+        if (p.out_bufs == 1 || p.stages >= std::min(3, loads)) break;
+    }
     const long long n_work = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n * p.n_tiles_n;
     if (n_work > 0x7fffffffLL) return DLF_E_UNSUPPORTED;
     p.n_work = static_cast<int>(n_work);
@@ -411,7 +490,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     p.bias = a.bias; p.res = static_cast<const __half*>(a.res); p.out = static_cast<__half*>(a.y);
     p.status = status_dev;
 
-    CUtensorMap tmx, tmw, tmy;
+    CUtensorMap tmx, tmw, tmy, tmr;
     const uint64_t taps64 = static_cast<uint64_t>(a.kh) * a.kw;
     if (p.grouped) {
         // input seen as (64 channels, W, H, N, C_in / 64): one box carries kg chunks of a tap's window
@@ -458,10 +537,15 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         const uint32_t es[4] = {1, 1, 1, 1};
         int rc = encode_tmap(&tmy, a.y, 4, dims, strides, box, es);
         if (rc) return rc;
+        tmr = tmy;
+        if (a.res && !a.pool) {   // the residual has the output's shape
+            rc = encode_tmap(&tmr, a.res, 4, dims, strides, box, es);
+            if (rc) return rc;
+        }
     }
     const int grid = std::max(1, std::min(sm_count, p.n_work));
     const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024, 120 * 1024);
-    cudaError_t e = launch_kernel(pick_kernel(a.act, a.pool != 0, a.res != nullptr), grid, kThreads, smem, s, tmx, tmw, tmy, p);
+    cudaError_t e = launch_kernel(pick_kernel(a.act, a.pool != 0, a.res != nullptr), grid, kThreads, smem, s, tmx, tmw, tmy, tmr, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 
