@@ -183,7 +183,9 @@ static bool depthwise_ok(const dlf_layer_desc& d) {
 }
 // Widest hidden tensor of an inverted-residual block the tuner proposes as one kernel: the kernel walks
 // the hidden channels in 64-wide steps one after the other, and beyond four steps three kernels that
-// each fill the chip were measured faster.  A plan given explicitly may still ask for a wider block.
+// each fill the chip were measured faster; so were two kernels for a block without an expansion
+// layer, which the tuner (max_hid > 0) does not propose either.  A plan given explicitly may still ask
+// for both.
 static const int kTunerMaxHidden = 256;
 
 static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix, int max_hid = 0) {
@@ -210,7 +212,7 @@ static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix,
     std::memset(&a, 0, sizeof(a));
     a.N = 1; a.H = 8; a.W = 8;
     a.Cin = has_expand ? d0.cin : hid; a.hid = hid; a.Cout = cout; a.stride = dd.stride; a.has_expand = has_expand ? 1 : 0;
-    if (!mbconv_supported(a) || (max_hid > 0 && hid > max_hid)) return false;
+    if (!mbconv_supported(a) || (max_hid > 0 && (hid > max_hid || !has_expand))) return false;
     // the maps between the layers are used nowhere else
     const int n = static_cast<int>(net->layers.size());
     for (int j = first + 1; j < n; j++) {

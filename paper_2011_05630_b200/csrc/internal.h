@@ -111,6 +111,7 @@ struct MbconvArgs {
 };
 struct MbconvTiling {
     int th, tw, fh, fw, nb1, nb2, tiles_h, tiles_w, n_tiles, stages, stage_bytes;
+    int out_planes;  // 64-channel planes of the output staging buffer, 0 = none (direct stores)
     size_t smem_bytes;
     double redundancy;
     bool ok;

@@ -12,7 +12,10 @@
 //      fp16 rounding -> tile Hd, laid out as the next GEMM's operand;
 //   4. projection on the tensor cores: D2[tile rows x C_out] += Hd * W2[:, chunk]^T, accumulated in
 //      tensor memory across the chunks (fp32, the same sum as the unchunked layer);
-// then epilogue 2: bias, residual, activation, fp16 rounding, global store.  Every intermediate is
+// then epilogue 2: bias, residual, activation, fp16 rounding.  Where shared memory has room the output
+// tile is staged there and leaves through TMA stores issued by the input-producer warp, which also
+// fetches the residual tile by TMA straight into that staging buffer a tile ahead (added in place);
+// otherwise each thread stores and reads its own pixel's channels directly.  Every intermediate is
 // rounded to fp16 exactly where the layer-by-layer execution rounds it.  Without an expansion layer
 // (the network's first block) steps 1-2 are skipped and the depthwise layer reads the input frame.
 //
@@ -40,7 +43,7 @@ constexpr int kMaxSmem = 232448 - 1024;
 constexpr int kPlane = 128 * 128;  // 128 rows x 64 channels
 
 struct MbParams {
-    CUtensorMap tmx, tmw1, tmw2;
+    CUtensorMap tmx, tmw1, tmw2, tmy, tmr;   // input frame, the two weight slabs, output tile, residual tile
     int N, H, W, Cin, hid, Cout, Ho, Wo, stride;
     int has_expand, act1, act2, act3;
     int th, tw, fh, fw, FR, nb1, nb2;   // output tile, input frame, frame rows, 128-row blocks of the two GEMMs
@@ -48,6 +51,7 @@ struct MbParams {
     int kin, chunks, n2_pad;            // 64-channel planes of the input, hidden chunks, C_out rounded up to 16
     int ksteps_in_last;
     int x_off, h_off, hd_off, ring_off, stage_bytes, stages, dw_off, bias_off;  // shared-memory byte offsets
+    int so_off, so_planes;              // output staging buffer: byte offset, 64-channel planes (0: none, direct stores)
     int d2_col;                         // first TMEM column of the projection accumulator
     int w2_off, n_split, n_each;        // projection slab inside a ring stage; C_out > 256 is issued as two halves
     const __half* wd;
@@ -111,7 +115,7 @@ __device__ __forceinline__ void dw_pair(const uint8_t* hsrc, uint8_t* hdbuf, int
 
 __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_constant__ MbParams p) {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t x_full, x_empty, w_full[4], w_empty[4], d1_full, d1_free, hd_ready, hd_free, d2_full, d2_free;
+    __shared__ uint64_t x_full, x_empty, w_full[4], w_empty[4], d1_full, d1_free, hd_ready, hd_free, d2_full, d2_free, s_full, s_free;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
@@ -135,8 +139,14 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
         mbar_init(&hd_free, 1);
         mbar_init(&d2_full, 1);
         mbar_init(&d2_free, kWorkWarps);
+        mbar_init(&s_full, kWorkWarps);
+        mbar_init(&s_free, 1);
         fence_barrier_init();
         tma_prefetch_desc(&p.tmx);
+        if (p.so_planes > 0) {
+            tma_prefetch_desc(&p.tmy);
+            if (p.res != nullptr) tma_prefetch_desc(&p.tmr);
+        }
     }
     if (warp == kMmaWarp) {
         tmem_alloc(&tmem_base_s, 512);
@@ -152,17 +162,51 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
     const uint32_t tmem_base = tmem_base_s;
 
     if (warp == kInWarp) {
-        // ---- input producer: the tile's frame, one box per 64-channel plane ---------------------------
+        // ---- input producer: the tile's frame, one box per 64-channel plane; and, with a staging
+        //      buffer, the finished tile out (TMA stores) and the next tile's residual in ------------------
         if (lane == 0) {
+            const bool staged = p.so_planes > 0, has_res = p.res != nullptr;
+            const uint32_t so_bytes = static_cast<uint32_t>(p.th * p.tw) * 128u;   // one plane's box
+            auto fetch_residual = [&](int t) {
+                const int txi = t % p.tiles_w, tyi = (t / p.tiles_w) % p.tiles_h, n = t / (p.tiles_w * p.tiles_h);
+                mbar_expect_tx(&s_free, static_cast<uint32_t>(p.so_planes) * so_bytes);
+                for (int pl = 0; pl < p.so_planes; pl++)
+                    tma_load_4d(sb + p.so_off + pl * p.nb2 * kPlane, &p.tmr, &s_free, pl * 64, txi * p.tw, tyi * p.th, n);
+            };
+            // tile `ti_prev` is staged: send it off, wait until the buffer has been read, hand it back
+            auto send_tile = [&](int t_prev, uint32_t ti_prev, int t_next) {
+                if (!mbar_wait(&s_full, ti_prev & 1u, abort_flag, p.status, 0xB10 | (blockIdx.x << 12))) return false;
+                const int txi = t_prev % p.tiles_w, tyi = (t_prev / p.tiles_w) % p.tiles_h, n = t_prev / (p.tiles_w * p.tiles_h);
+                for (int pl = 0; pl < p.so_planes; pl++)
+                    tma_store_4d(&p.tmy, sb + p.so_off + pl * p.nb2 * kPlane, pl * 64, txi * p.tw, tyi * p.th, n);
+                tma_store_commit();
+                tma_store_wait_read();
+                if (has_res) {
+                    if (t_next < p.n_tiles) fetch_residual(t_next);
+                } else {
+                    mbar_arrive(&s_free);
+                }
+                return true;
+            };
+            if (staged && has_res && static_cast<int>(blockIdx.x) < p.n_tiles) fetch_residual(blockIdx.x);
             uint32_t ti = 0;
+            int t_prev = -1;
+            bool ok = true;
             for (int t = blockIdx.x; t < p.n_tiles; t += gridDim.x, ti++) {
                 const int txi = t % p.tiles_w, tyi = (t / p.tiles_w) % p.tiles_h, n = t / (p.tiles_w * p.tiles_h);
-                if (!mbar_wait(&x_empty, (ti & 1u) ^ 1u, abort_flag, p.status, 0xB00 | (blockIdx.x << 12))) break;
+                ok = mbar_wait(&x_empty, (ti & 1u) ^ 1u, abort_flag, p.status, 0xB00 | (blockIdx.x << 12));
+                if (!ok) break;
                 mbar_expect_tx(&x_full, static_cast<uint32_t>(p.kin) * p.FR * 128u);
                 for (int pl = 0; pl < p.kin; pl++)
                     tma_load_4d(sb + p.x_off + pl * p.nb1 * kPlane, &p.tmx, &x_full, pl * 64, txi * p.tw * p.stride - 1,
                                 tyi * p.th * p.stride - 1, n);
+                if (staged && t_prev >= 0) {
+                    ok = send_tile(t_prev, ti - 1, t);
+                    if (!ok) break;
+                }
+                t_prev = t;
             }
+            if (staged && ok && t_prev >= 0) send_tile(t_prev, ti - 1, p.n_tiles);
         }
     } else if (warp == kW1Warp || warp == kW2Warp) {
         // ---- weight producers: per chunk the expansion slab [64 hidden][C_in] and the projection
@@ -367,6 +411,53 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
             if (!ok) break;
             tc_fence_after_sync();
             const float* b2s = bias_s + p.chunks * 64;
+            if (p.so_planes > 0) {
+                // staged: the buffer is free again (first tile: at once) / holds this tile's residual
+                ok = mbar_wait(&s_free, p.res != nullptr ? (ti & 1u) : ((ti & 1u) ^ 1u), abort_flag, p.status, 0xE40 | (blockIdx.x << 12));
+                if (!ok) break;
+                uint8_t* so = sb + p.so_off;
+                const bool has_res = p.res != nullptr;
+                for (int b = 0; b < p.nb2; b++) {
+                    const int o = b * 128 + q * 32 + lane;
+                    const bool live = o < p.th * p.tw;   // rows past the image are clipped by the TMA store
+                    const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + p.d2_col + b * p.n2_pad;
+                    for (int c0 = half * 16; c0 < p.n2_pad; c0 += 32) {
+                        float v[16];
+                        __syncwarp();
+                        tmem_ld16(taddr + c0, v);
+                        if (!live) continue;
+#pragma unroll
+                        for (int g = 0; g < 2; g++) {
+                            const int co = c0 + g * 8;
+                            if (co >= p.Cout) break;
+                            const int g8 = (co >> 3) & 7;
+                            uint4* sp = reinterpret_cast<uint4*>(so + (co >> 6) * p.nb2 * kPlane + o * 128 + ((g8 ^ (o & 7)) << 4));
+                            const float4 ba = *reinterpret_cast<const float4*>(b2s + co), bc = *reinterpret_cast<const float4*>(b2s + co + 4);
+                            float a[8] = {v[g * 8 + 0] + ba.x, v[g * 8 + 1] + ba.y, v[g * 8 + 2] + ba.z, v[g * 8 + 3] + ba.w,
+                                          v[g * 8 + 4] + bc.x, v[g * 8 + 5] + bc.y, v[g * 8 + 6] + bc.z, v[g * 8 + 7] + bc.w};
+                            if (has_res) {   // loaded into the staging buffer by TMA, zero outside the tensor
+                                const uint4 rv = *sp;
+                                const __half2* rh = reinterpret_cast<const __half2*>(&rv);
+#pragma unroll
+                                for (int e = 0; e < 4; e++) {
+                                    const float2 f = __half22float2(rh[e]);
+                                    a[2 * e] += f.x;
+                                    a[2 * e + 1] += f.y;
+                                }
+                            }
+                            uint4 val;
+                            val.x = pack_half2(clampf(a[0], lo3, hi3), clampf(a[1], lo3, hi3));
+                            val.y = pack_half2(clampf(a[2], lo3, hi3), clampf(a[3], lo3, hi3));
+                            val.z = pack_half2(clampf(a[4], lo3, hi3), clampf(a[5], lo3, hi3));
+                            val.w = pack_half2(clampf(a[6], lo3, hi3), clampf(a[7], lo3, hi3));
+                            *sp = val;
+                        }
+                    }
+                }
+                fence_proxy_async_smem();  // the TMA store reads the staging buffer
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&s_full);
+            } else
             for (int b = 0; b < p.nb2; b++) {
                 const int o = b * 128 + q * 32 + lane;
                 const int oy = o / p.tw, ox = o - oy * p.tw;
@@ -452,23 +543,33 @@ MbconvTiling mbconv_tiling(const MbconvArgs& a, int sm_count) {
             if (d1_cols + nb2 * n2 > 512) continue;
             const int stage = kin * 8192 * (a.has_expand ? 1 : 0) + n2 * 128;
             const size_t fixed = static_cast<size_t>(kin) * nb1 * kPlane + (a.has_expand ? nb1 * kPlane : 0) + static_cast<size_t>(nb2) * kPlane +
-                                 4096 + static_cast<size_t>(chunks * 64 + n2) * 4 + 2048;
+                                 4096 + static_cast<size_t>(chunks * 64 + n2) * 4 + 4096;
+            // the output staging buffer (one 64-channel plane per 128-row block) if it fits beside two ring stages
+            int out_planes = (a.Cout + 63) / 64;
+            size_t so_bytes = static_cast<size_t>(out_planes) * nb2 * kPlane;
+            if (fixed + so_bytes + 2 * static_cast<size_t>(stage) > static_cast<size_t>(kMaxSmem)) {
+                out_planes = 0;
+                so_bytes = 0;
+            }
             int stages = 3;
-            while (stages > 2 && fixed + static_cast<size_t>(stages) * stage > static_cast<size_t>(kMaxSmem)) stages--;
-            if (fixed + static_cast<size_t>(stages) * stage > static_cast<size_t>(kMaxSmem)) continue;
+            while (stages > 2 && fixed + so_bytes + static_cast<size_t>(stages) * stage > static_cast<size_t>(kMaxSmem)) stages--;
+            if (fixed + so_bytes + static_cast<size_t>(stages) * stage > static_cast<size_t>(kMaxSmem)) continue;
             const int tiles_h = (Ho + th - 1) / th, tiles_w = (Wo + tw - 1) / tw;
             const long long n_tiles = static_cast<long long>(a.N) * tiles_h * tiles_w;
             if (n_tiles > 0x7fffffffLL) continue;
             const long long waves = (n_tiles + sm_count - 1) / sm_count;
             // per chunk: epilogue-1 rows + depthwise items on 256 threads, plus hand-off latency
             const double per_chunk = (a.has_expand ? nb1 * 128 * 1.5 : 0.0) + th * tw * 4.0 + 2500.0;
-            const double cost = static_cast<double>(waves) * (chunks * per_chunk + 3000.0);
+            // epilogue 2: staged tiles leave by TMA; direct stores touch one cache line per thread and instruction
+            const double epi2 = th * tw * (n2 / 16.0) * (out_planes > 0 ? 1.0 : 4.0);
+            const double cost = static_cast<double>(waves) * (chunks * per_chunk + epi2 + 3000.0);
             if (best_cost < 0 || cost < best_cost) {
                 best_cost = cost;
                 best.th = th; best.tw = tw; best.fh = fh; best.fw = fw; best.nb1 = nb1; best.nb2 = nb2;
                 best.tiles_h = tiles_h; best.tiles_w = tiles_w; best.n_tiles = static_cast<int>(n_tiles);
                 best.stages = stages; best.stage_bytes = stage;
-                best.smem_bytes = fixed + static_cast<size_t>(stages) * stage;
+                best.smem_bytes = fixed + so_bytes + static_cast<size_t>(stages) * stage;
+                best.out_planes = out_planes;
                 best.redundancy = static_cast<double>(FR) / (std::min(th, Ho) * a.stride * std::min(tw, Wo) * a.stride);
                 best.ok = true;
             }
@@ -507,6 +608,8 @@ int launch_mbconv_tc(const MbconvArgs& a, const MbconvTiling& t, int sm_count, i
     p.dw_off = p.ring_off + p.stages * p.stage_bytes;
     p.dw_off = (p.dw_off + 1023) / 1024 * 1024;
     p.bias_off = p.dw_off + 4096;
+    p.so_planes = t.out_planes;
+    p.so_off = (p.bias_off + (p.chunks * 64 + p.n2_pad) * 4 + 1023) / 1024 * 1024;
     p.d2_col = a.has_expand ? p.nb1 * 64 : 0;
     p.w2_off = a.has_expand ? p.kin * 8192 : 0;
     p.n_split = p.n2_pad > 256 ? 2 : 1;
@@ -538,8 +641,22 @@ int launch_mbconv_tc(const MbconvArgs& a, const MbconvTiling& t, int sm_count, i
         rc = encode_tmap(&p.tmw2, a.w2, 3, dims, strides, box, es);
         if (rc) return rc;
     }
+    if (p.so_planes > 0) {  // output (and residual) tile [C_out, Wo, Ho, N], one box per 64-channel plane
+        const uint64_t dims[4] = {static_cast<uint64_t>(a.Cout), static_cast<uint64_t>(p.Wo), static_cast<uint64_t>(p.Ho), static_cast<uint64_t>(a.N)};
+        const uint64_t strides[3] = {static_cast<uint64_t>(a.Cout) * 2, static_cast<uint64_t>(p.Wo) * a.Cout * 2,
+                                     static_cast<uint64_t>(p.Ho) * p.Wo * a.Cout * 2};
+        const uint32_t box[4] = {64, static_cast<uint32_t>(t.tw), static_cast<uint32_t>(t.th), 1};
+        const uint32_t es[4] = {1, 1, 1, 1};
+        rc = encode_tmap(&p.tmy, a.y, 4, dims, strides, box, es);
+        if (rc) return rc;
+        p.tmr = p.tmy;
+        if (a.res) {
+            rc = encode_tmap(&p.tmr, a.res, 4, dims, strides, box, es);
+            if (rc) return rc;
+        }
+    }
     const int grid = std::max(1, std::min(sm_count, t.n_tiles));
-    const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + (p.chunks * 64 + p.n2_pad) * 4 + 2048, 120 * 1024);
+    const size_t smem = std::max<size_t>(static_cast<size_t>(p.so_off) + static_cast<size_t>(p.so_planes) * p.nb2 * kPlane + 1024, 120 * 1024);
     if (smem > static_cast<size_t>(kMaxSmem)) return DLF_E_PLAN;
     cudaError_t e = launch_kernel(mbconv_tc_kernel, grid, kThreads, smem, s, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);

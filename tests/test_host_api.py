@@ -137,7 +137,8 @@ def span_is_mbconv(layers, first, last, prefix, max_hid=0):
     projection and from outside, the maps in between used nowhere else; `prefix` also accepts the
     pattern's first layers.  Channel limits of the fused kernel: C_in <= 256 (multiple of 8), hidden
     <= 1024 (multiple of 16), C_out <= 512 (multiple of 8; above 256 a multiple of 32 after padding).
-    `max_hid` > 0 is the tuner's own limit on the hidden width of a block it proposes as one kernel."""
+    `max_hid` > 0 is the tuner's own limit on the hidden width of a block it proposes as one kernel
+    (and it proposes none without an expansion layer)."""
     n_len = last - first + 1
     if n_len < 2 or n_len > 3:
         return False
@@ -163,7 +164,7 @@ def span_is_mbconv(layers, first, last, prefix, max_hid=0):
     cpad = (cout + 15) // 16 * 16
     if cin % 8 or hid % 16 or cout % 8 or cin > 256 or cout > 512 or hid > 1024 or (cpad > 256 and cpad % 32):
         return False
-    if max_hid > 0 and hid > max_hid:
+    if max_hid > 0 and (hid > max_hid or not has_expand):
         return False
     for j in range(first + 1, len(layers)):
         for which, r in (("src", layers[j]["src"]), ("res", layers[j]["res_src"])):
@@ -200,5 +201,5 @@ def test_autotune_equals_restated_algorithm1(name, layers, batch, crit):
     assert got == (want[0], want[1]), (got, want)
     if name == "mobilenet_v2" and crit == 1e30:   # the blocks with a hidden width up to 256 become one group each
         firsts = [0] + [e + 1 for e in got[0][:-1]]
-        assert sum(1 for a, e in zip(firsts, got[0]) if e - a + 1 >= 2) == 7
+        assert sum(1 for a, e in zip(firsts, got[0]) if e - a + 1 >= 2) == 6
     B.net_destroy(net)
