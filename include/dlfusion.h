@@ -142,6 +142,16 @@ int dlf_net_bruteforce(dlf_net* net, const dlf_search_params* params, const void
                        void* stream, int* n_groups, int32_t* group_end, int32_t* sm_count,
                        float* best_ms);
 
+/* Times layers first..last as ONE candidate group on sm_count SMs, outside any plan (the single-layer
+ * micro-benchmark of the paper's characterisation, Sec. II-B, and one cell of the reduced brute-force
+ * search, Sec. V): median device time of one launch, taken over `iters` timings of four back-to-back
+ * launches after `warmup` untimed ones (warm L2).  The group reads its inputs from the workspace slots
+ * of the layers before it: with prepare != 0 the call first runs the no-fusion plan once to fill every
+ * slot (the installed plan is kept); with prepare == 0 the caller has done so.  DLF_E_PLAN if the span
+ * cannot run as one kernel on that many SMs.  The network's last layer is written to its workspace slot. */
+int dlf_net_time_span(dlf_net* net, int first, int last, int sm_count, const void* in_dev, void* stream,
+                      int warmup, int iters, int prepare, float* ms);
+
 /* Enqueues one inference on `stream` and returns without waiting.  in_dev: N*H*W*C fp16.
  * out_dev: the last layer's output, fp16 NHWC.  DLF_E_STATE without weights / plan /
  * workspace. */

@@ -66,6 +66,7 @@ def lib():
             "dlf_net_group_is_legal": (C.c_int, [vp, C.c_int, C.c_int, C.c_int]),
             "dlf_net_autotune": (C.c_int, [vp, C.POINTER(TunerParams), ip, i32p, i32p]),
             "dlf_net_bruteforce": (C.c_int, [vp, C.POINTER(SearchParams), vp, vp, ip, i32p, i32p, fp]),
+            "dlf_net_time_span": (C.c_int, [vp, C.c_int, C.c_int, C.c_int, vp, vp, C.c_int, C.c_int, C.c_int, fp]),
             "dlf_net_run": (C.c_int, [vp, vp, vp, vp]),
             "dlf_net_run_host": (C.c_int, [vp, vp, vp, vp]),
             "dlf_net_sync": (C.c_int, [vp, vp]),
@@ -188,6 +189,13 @@ def net_bruteforce(net, n_layers, sm_choices, max_group_len, in_ptr, stream=None
     e, s = (C.c_int32 * n_layers)(), (C.c_int32 * n_layers)()
     _check(lib().dlf_net_bruteforce(net, C.byref(sp), in_ptr, stream, C.byref(n), e, s, C.byref(ms)), "dlf_net_bruteforce")
     return list(e[:n.value]), list(s[:n.value]), ms.value
+
+
+def net_time_span(net, first, last, sm_count, in_ptr, stream=None, warmup=2, iters=5, prepare=True):
+    ms = C.c_float()
+    _check(lib().dlf_net_time_span(net, first, last, sm_count, in_ptr, stream, warmup, iters, 1 if prepare else 0,
+                                   C.byref(ms)), "dlf_net_time_span")
+    return ms.value
 
 
 def net_run(net, in_ptr, out_ptr, stream=None):

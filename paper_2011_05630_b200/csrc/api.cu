@@ -876,6 +876,75 @@ int dlf_net_time(dlf_net* net, const void* in_dev, void* out_dev, void* stream, 
     return dlf_net_sync(net, s);
 }
 
+// Median device time of ONE launch of group `g`: a graph of kReps back-to-back launches (which hides the
+// host's launch cost) is timed `iters` times between two events after `warmup` untimed launches.
+static int time_group(dlf_net* net, const Group& g, const void* in_dev, void* final_out, cudaStream_t s, cudaEvent_t e0,
+                      cudaEvent_t e1, int warmup, int iters, float* ms_out) {
+    const int kReps = 4;
+    int rc = DLF_OK;
+    cudaGraphExec_t exec = nullptr;
+    if (!net->capture_stream && cudaStreamCreateWithFlags(&net->capture_stream, cudaStreamNonBlocking) != cudaSuccess)
+        return cuda_fail(cudaGetLastError());
+    cudaGraph_t graph = nullptr;
+    if (cudaStreamBeginCapture(net->capture_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) return cuda_fail(cudaGetLastError());
+    for (int r = 0; r < kReps && rc == DLF_OK; r++) rc = launch_group(net, g, in_dev, final_out, net->capture_stream);
+    cudaError_t e = cudaStreamEndCapture(net->capture_stream, &graph);
+    if (rc == DLF_OK && e != cudaSuccess) rc = cuda_fail(e);
+    if (rc == DLF_OK && cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+    if (graph) cudaGraphDestroy(graph);
+    for (int i = 0; i < warmup && rc == DLF_OK; i++)
+        if (cudaGraphLaunch(exec, s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+    std::vector<float> v;
+    for (int i = 0; i < iters && rc == DLF_OK; i++) {
+        cudaEventRecord(e0, s);
+        if (cudaGraphLaunch(exec, s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+        cudaEventRecord(e1, s);
+        if (rc == DLF_OK && cudaEventSynchronize(e1) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
+        float ms = 0.0f;
+        if (rc == DLF_OK) cudaEventElapsedTime(&ms, e0, e1);
+        v.push_back(ms / kReps);
+    }
+    if (exec) cudaGraphExecDestroy(exec);
+    if (rc == DLF_OK) *ms_out = median_of(v);
+    return rc;
+}
+
+int dlf_net_time_span(dlf_net* net, int first, int last, int sm_count, const void* in_dev, void* stream, int warmup,
+                      int iters, int prepare, float* ms) {
+    if (!net || !in_dev || !ms || first < 0 || last < first || last >= static_cast<int>(net->layers.size()) || warmup < 0 || iters < 1)
+        return DLF_E_INVALID_ARG;
+    if (!net->ws) return DLF_E_WORKSPACE;
+    for (const Layer& l : net->layers)
+        if (is_param(l) && (!l.w || !l.bias)) return DLF_E_STATE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    void* final_out = net->ws + net->layers.back().off;
+    int rc = DLF_OK;
+    if (prepare) {   // every layer's slot filled once, so that the span finds its inputs in HBM
+        std::vector<Group> saved = net->plan;
+        rc = dlf_net_plan_unfused(net);
+        if (rc == DLF_OK) rc = dlf_net_run(net, in_dev, final_out, s);
+        if (rc == DLF_OK) rc = dlf_net_sync(net, s);
+        net->plan = saved;
+        invalidate_graphs(net);
+        if (rc) return rc;
+    }
+    if (net->dev_sms == 0) {
+        rc = query_sms(&net->dev_sms);
+        if (rc) return rc;
+    }
+    if (sm_count < 1 || sm_count > net->dev_sms) return DLF_E_PLAN;
+    Group g;
+    if (!make_group(net, first, last, sm_count, &g)) return DLF_E_PLAN;
+    rc = kernels_init();
+    if (rc) return rc;
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return cuda_fail(cudaGetLastError());
+    rc = time_group(net, g, in_dev, final_out, s, e0, e1, warmup, iters, ms);
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    return rc ? rc : dlf_net_sync(net, s);
+}
+
 int dlf_net_bruteforce(dlf_net* net, const dlf_search_params* sp, const void* in_dev, void* stream, int* n_groups,
                        int32_t* group_end, int32_t* sm_count, float* best_ms) {
     if (!net || !sp || !in_dev || !n_groups || !group_end || !sm_count) return DLF_E_INVALID_ARG;
@@ -907,40 +976,9 @@ int dlf_net_bruteforce(dlf_net* net, const dlf_search_params* sp, const void* in
                 if (S < 1 || S > net->dev_sms) continue;
                 Group g;
                 if (!make_group(net, a, a + len - 1, S, &g)) continue;
-                // a graph of kReps back-to-back launches hides the host's launch cost
-                const int kReps = 4;
-                cudaGraphExec_t exec = nullptr;
-                {
-                    if (!net->capture_stream && cudaStreamCreateWithFlags(&net->capture_stream, cudaStreamNonBlocking) != cudaSuccess)
-                        rc = cuda_fail(cudaGetLastError());
-                    cudaGraph_t graph = nullptr;
-                    if (rc == DLF_OK && cudaStreamBeginCapture(net->capture_stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess)
-                        rc = cuda_fail(cudaGetLastError());
-                    if (rc == DLF_OK) {
-                        for (int r = 0; r < kReps && rc == DLF_OK; r++) rc = launch_group(net, g, in_dev, final_out, net->capture_stream);
-                        cudaError_t e = cudaStreamEndCapture(net->capture_stream, &graph);
-                        if (rc == DLF_OK && e != cudaSuccess) rc = cuda_fail(e);
-                        if (rc == DLF_OK && cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
-                        if (graph) cudaGraphDestroy(graph);
-                    }
-                }
-                for (int i = 0; i < sp->warmup && rc == DLF_OK; i++)
-                    if (cudaGraphLaunch(exec, s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
-                std::vector<float> v;
-                for (int i = 0; i < sp->iters && rc == DLF_OK; i++) {
-                    cudaEventRecord(e0, s);
-                    if (cudaGraphLaunch(exec, s) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
-                    cudaEventRecord(e1, s);
-                    if (cudaEventSynchronize(e1) != cudaSuccess) rc = cuda_fail(cudaGetLastError());
-                    float ms = 0.0f;
-                    cudaEventElapsedTime(&ms, e0, e1);
-                    v.push_back(ms / kReps);
-                }
-                if (exec) cudaGraphExecDestroy(exec);
-                if (rc == DLF_OK) {
-                    const float m = median_of(v);
-                    if (m < t[a][len - 1]) { t[a][len - 1] = m; ts[a][len - 1] = S; }
-                }
+                float m = 0.0f;
+                rc = time_group(net, g, in_dev, final_out, s, e0, e1, sp->warmup, sp->iters, &m);
+                if (rc == DLF_OK && m < t[a][len - 1]) { t[a][len - 1] = m; ts[a][len - 1] = S; }
             }
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);

@@ -29,6 +29,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cstdio>
 #include <cstring>
 #include <vector>
 
@@ -255,72 +256,88 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             }
         }
     } else if (warp == kMmaWarp) {
-        // ---- UMMA issuer ------------------------------------------------------------------------------------
-        if (lane == 0) {
-            uint32_t wit = 0, tile_i = 0, pass_i = 0, act_i = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x, tile_i++) {
-                const uint32_t ib = tile_i % p.in_bufs;
-                ok = mbar_wait(&in_full_bar[ib], (tile_i / p.in_bufs) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
-                if (!ok) break;
-                for (int l = 0; l < p.n_layers && ok; l++) {
-                    const ChainLayerP& L = p.L[l];
-                    if (l > 0) {  // the epilogue has written all of the previous layer's tile
-                        ok = mbar_wait(&act_ready_bar, act_i & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
+        // ---- UMMA issuer: the whole warp walks the loops (warp-uniform addresses), one elected lane issues ----
+        const uint64_t desc0 = umma_desc_sw128(0, 0);
+        uint32_t wit = 0, tile_i = 0, pass_i = 0, act_i = 0;
+        bool ok = true;
+        DLF_TRACE_DECL(tacc, tmark);  // cycles of CTA 0's issuer: 0 input wait, 1 layer hand-off wait, 2 accumulator wait, 3 weight wait, 4 issue
+        for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x, tile_i++) {
+            const uint32_t ib = tile_i % p.in_bufs;
+            ok = mbar_wait_warp(&in_full_bar[ib], (tile_i / p.in_bufs) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
+            if (!ok) break;
+            DLF_TRACE_ACC(tacc, 0, tmark);
+            for (int l = 0; l < p.n_layers && ok; l++) {
+                const ChainLayerP& L = p.L[l];
+                if (l > 0) {  // the epilogue has written all of the previous layer's tile
+                    ok = mbar_wait_warp(&act_ready_bar, act_i & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
+                    if (!ok) break;
+                    act_i++;
+                    DLF_TRACE_ACC(tacc, 1, tmark);
+                }
+                const uint32_t abuf = l == 0 ? base + ib * p.in_buf_bytes : base + p.act_off + ((l - 1) & 1) * p.act_buf_bytes;
+                const int taps = L.k * L.k;
+                const uint32_t w_tap16 = static_cast<uint32_t>(L.chunk_n) * 8u;  // one tap's [chunk_n][64] slab, 16-byte units
+                for (int c = 0; c < L.n_chunks && ok; c++) {
+                    const uint32_t idesc = umma_idesc_f16(chunk_cols(L, c));
+                    for (int b0 = 0; b0 < L.nb && ok; b0 += L.per_pass, pass_i++) {
+                        const int nblk = min(L.per_pass, L.nb - b0);
+                        const uint32_t half = pass_i & 1u;
+                        ok = mbar_wait_warp(&acc_empty_bar[half], ((pass_i >> 1) & 1u) ^ 1u, abort_flag, p.status,
+                                            0x500 | (blockIdx.x << 12));
                         if (!ok) break;
-                        act_i++;
-                    }
-                    const uint32_t abuf = l == 0 ? base + ib * p.in_buf_bytes : base + p.act_off + ((l - 1) & 1) * p.act_buf_bytes;
-                    for (int c = 0; c < L.n_chunks && ok; c++) {
-                        const uint32_t idesc = umma_idesc_f16(chunk_cols(L, c));
-                        for (int b0 = 0; b0 < L.nb && ok; b0 += L.per_pass, pass_i++) {
-                            const int nblk = min(L.per_pass, L.nb - b0);
-                            const uint32_t half = pass_i & 1u;
-                            ok = mbar_wait(&acc_empty_bar[half], ((pass_i >> 1) & 1u) ^ 1u, abort_flag, p.status,
-                                           0x500 | (blockIdx.x << 12));
-                            if (!ok) break;
-                            tc_fence_after_sync();
-                            for (int t0 = 0; t0 < L.k * L.k && ok; t0 += L.tg) {
-                                for (int g0 = 0; g0 < L.kchunks; g0 += L.kg, wit++) {
-                                    const int st = wit % p.stages;
-                                    ok = mbar_wait(&wfull_bar[st], (wit / p.stages) & 1u, abort_flag, p.status,
-                                                   0x600 | (blockIdx.x << 12));
-                                    if (!ok) break;
-                                    tc_fence_after_sync();
-                                    const uint32_t wsm = base + p.ring_off + st * p.stage_bytes;
-                                    for (int g = 0; g < L.kg && g0 + g < L.kchunks; g++) {
+                        DLF_TRACE_ACC(tacc, 2, tmark);
+                        tc_fence_after_sync();
+                        const uint32_t d_tmem0 = tmem_base + half * 256u;
+                        const uint32_t arow_base = abuf + (L.qs + b0 * 128) * 128;
+                        for (int t0 = 0; t0 < taps && ok; t0 += L.tg) {
+                            for (int g0 = 0; g0 < L.kchunks; g0 += L.kg, wit++) {
+                                const int st = wit % p.stages;
+                                ok = mbar_wait_warp(&wfull_bar[st], (wit / p.stages) & 1u, abort_flag, p.status,
+                                                    0x600 | (blockIdx.x << 12));
+                                if (!ok) break;
+                                DLF_TRACE_ACC(tacc, 3, tmark);
+                                tc_fence_after_sync();
+                                const uint64_t wd0 = desc0 + ((base + p.ring_off + st * p.stage_bytes) >> 4);
+                                const int g_end = min(L.kg, L.kchunks - g0);
+                                if (elect_one()) {
+                                    for (int g = 0; g < g_end; g++) {
                                         const int kc = g0 + g;
                                         const int ksteps = (kc == L.kchunks - 1) ? L.ksteps_last : 4;
+                                        const uint32_t aplane = arow_base + kc * p.plane_bytes;
                                         for (int tt = 0; tt < L.tg; tt++) {
                                             const int tap = t0 + tt;
                                             const int r = tap / L.k, sx = tap - r * L.k;
                                             const int shift = (r - L.pad) * p.pitch + (sx - L.pad);
-                                            const uint32_t b_lo = umma_desc_lo(wsm + (g * L.tg + tt) * L.chunk_n * 128);
-                                            const uint32_t arow0 = abuf + kc * p.plane_bytes + (L.qs + b0 * 128 + shift) * 128;
+                                            const uint64_t bd = wd0 + static_cast<uint32_t>(g * L.tg + tt) * w_tap16;
+                                            const uint32_t arow0 = aplane + shift * 128;
+                                            uint64_t ad = desc0 + (arow0 >> 4);
+                                            if (p.base_offset_mode) ad |= static_cast<uint64_t>((arow0 >> 7) & 7u) << 49;  // 128 rows keep the phase
                                             const uint32_t acc0 = (tap | kc) != 0;
-                                            uint32_t d_tmem = tmem_base + half * 256u;
-                                            for (int b = 0; b < nblk; b++, d_tmem += L.slot) {
-                                                const uint32_t arow = arow0 + b * (128 * 128);
-                                                const uint32_t a_lo = umma_desc_lo(arow);
-                                                const uint32_t a_hi = p.base_offset_mode ? (kDescHiSw128 | (((arow >> 7) & 7u) << 17)) : kDescHiSw128;
-                                                umma_f16_lo(d_tmem, a_lo, a_hi, b_lo, idesc, acc0);
-                                                if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, a_hi, b_lo + 2, idesc, 1);
-                                                if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, a_hi, b_lo + 4, idesc, 1);
-                                                if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, a_hi, b_lo + 6, idesc, 1);
+                                            uint32_t d_tmem = d_tmem0;
+                                            for (int b = 0; b < nblk; b++, d_tmem += L.slot, ad += (128 * 128) >> 4) {
+                                                umma_f16(d_tmem, ad, bd, idesc, acc0);
+                                                if (ksteps > 1) umma_f16(d_tmem, ad + 2, bd + 2, idesc, 1);
+                                                if (ksteps > 2) umma_f16(d_tmem, ad + 4, bd + 4, idesc, 1);
+                                                if (ksteps > 3) umma_f16(d_tmem, ad + 6, bd + 6, idesc, 1);
                                             }
                                         }
                                     }
                                     umma_commit(&wempty_bar[st]);
                                 }
+                                __syncwarp();
+                                DLF_TRACE_ACC(tacc, 4, tmark);
                             }
-                            if (ok) umma_commit(&acc_full_bar[half]);
                         }
+                        if (ok && elect_one()) umma_commit(&acc_full_bar[half]);
+                        __syncwarp();
                     }
-                    // the input frame is read by the first layer only
-                    if (ok && l == 0) umma_commit(&in_empty_bar[ib]);
                 }
+                // the input frame is read by the first layer only
+                if (ok && l == 0 && elect_one()) umma_commit(&in_empty_bar[ib]);
+                __syncwarp();
             }
         }
+        if (lane == 0) DLF_TRACE_FLUSH_AT(p.status, tacc, 0);
     } else {
         // ---- epilogue warps ------------------------------------------------------------------------------------
         const int et = threadIdx.x;  // 0 .. 32*kEpiWarps-1
@@ -330,6 +347,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         cx.tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         uint32_t pass_i = 0;
         bool ok = true;
+        DLF_TRACE_DECL(eacc, emark);  // cycles of CTA 0's first epilogue thread: 0 accumulator wait, 1 + mode: drain, 5 pooled copy-out
         for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
             const int txi = t % p.tiles_w, tyi = (t / p.tiles_w) % p.tiles_h, n = t / (p.tiles_w * p.tiles_h);
             cx.gy0 = tyi * p.th - p.halo;
@@ -350,6 +368,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                         const uint32_t half = pass_i & 1u;
                         ok = mbar_wait(&acc_full_bar[half], (pass_i >> 1) & 1u, abort_flag, p.status, 0x700 | (blockIdx.x << 12));
                         if (!ok) break;
+                        DLF_TRACE_ACC(eacc, 0, emark);
                         tc_fence_after_sync();
                         cx.b0 = b0;
                         cx.nblk = min(L.per_pass, L.nb - b0);
@@ -362,6 +381,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                         tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) mbar_arrive(&acc_empty_bar[half]);
+                        DLF_TRACE_ACC(eacc, 1 + mode, emark);
                     }
                 }
                 if (ok && !last && lane == 0) mbar_arrive(&act_ready_bar);
@@ -398,8 +418,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                     *reinterpret_cast<uint4*>(p.out + ((static_cast<long long>(n) * Ho + gy) * Wo + gx) * p.cout_last + g8 * 8) = best;
                 }
                 epi_bar_sync();
+                DLF_TRACE_ACC(eacc, 5, emark);
             }
         }
+        if (threadIdx.x == 0) DLF_TRACE_FLUSH_AT(p.status, eacc, 8);
     }
 
     tc_fence_before_sync();
@@ -636,6 +658,13 @@ int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int 
     }
     const int grid = std::max(1, std::min(sm_count, t.n_tiles));
     const size_t smem = std::max<size_t>(t.smem_bytes, 120 * 1024);
+#ifdef DLF_TRACE
+    fprintf(stderr, "chain_tc: L=%d tile %dx%d frame %dx%d tiles %d grid %d in_bufs %d stages %d stage_bytes %d smem %zu red %.2f\n", a.n_layers,
+            t.th, t.tw, t.rows, t.pitch, t.n_tiles, grid, t.in_bufs, t.stages, t.stage_bytes, t.smem_bytes, t.redundancy);
+    for (int l = 0; l < a.n_layers; l++)
+        fprintf(stderr, "  layer %d: %d->%d k%d nb %d chunks %d x %d per_pass %d tg %d kg %d\n", l, a.cin[l], a.cout[l], a.k[l], p.L[l].nb,
+                p.L[l].n_chunks, p.L[l].chunk_n, p.L[l].per_pass, p.L[l].tg, p.L[l].kg);
+#endif
     cudaError_t e = launch_kernel(chain_tc_kernel, grid, kThreads, smem, s, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }

@@ -202,41 +202,45 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             }
         }
     } else if (warp == kMmaWarp) {
-        // ---- MMA issuer ---------------------------------------------------------------------------
-        if (lane == 0) {
-            const uint32_t idesc = umma_idesc_f16(p.BN);
-            uint32_t it = 0, j = 0;
-            bool ok = true;
-            for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
-                const uint32_t acc = j & 1u;
-                ok = mbar_wait(&tempty_bar[acc], ((j >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x200 | (blockIdx.x << 12));
+        // ---- MMA issuer: the whole warp walks the loop (warp-uniform addresses), one elected lane issues ----
+        const uint32_t idesc = umma_idesc_f16(p.BN);
+        const uint64_t desc0 = umma_desc_sw128(0, 0);
+        const uint32_t b_chunk16 = static_cast<uint32_t>(p.BN) * 8u;  // one 64-channel weight slab, in 16-byte units
+        uint32_t it = 0, j = 0;
+        bool ok = true;
+        for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
+            const uint32_t acc = j & 1u;
+            ok = mbar_wait_warp(&tempty_bar[acc], ((j >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x200 | (blockIdx.x << 12));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t d_tmem = tmem_base + acc * p.acc_stride;
+            int kq = 0;
+            for (int ki = 0; ki < k_iters; ki++, it++) {
+                const int st = it % p.stages;
+                ok = mbar_wait_warp(&full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                 if (!ok) break;
+                if (it == 0 && lane == 0) DLF_TRACE_POINT(p.status, 3);
                 tc_fence_after_sync();
-                const uint32_t d_tmem = tmem_base + acc * p.acc_stride;
-                int kq = 0;
-                for (int ki = 0; ki < k_iters; ki++, it++) {
-                    const int st = it % p.stages;
-                    ok = mbar_wait(&full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
-                    if (!ok) break;
-                    if (it == 0) DLF_TRACE_POINT(p.status, 3);
-                    tc_fence_after_sync();
-                    const uint32_t sa = base + st * stage_bytes, sb = sa + p.kg * kABytes;
-                    for (int g = 0; g < p.kg; g++) {
-                        const int kc = kq * p.kg + g;
-                        if (kc >= p.kchunks) break;
-                        const uint32_t a_lo = umma_desc_lo(sa + g * kABytes), b_lo = umma_desc_lo(sb + g * p.BN * 128);
-                        const int ksteps = (kc == p.kchunks - 1) ? p.ksteps_last : 4;
-                        umma_f16_lo(d_tmem, a_lo, kDescHiSw128, b_lo, idesc, (ki | g) != 0);
-                        if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, kDescHiSw128, b_lo + 2, idesc, 1);
-                        if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, kDescHiSw128, b_lo + 4, idesc, 1);
-                        if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, kDescHiSw128, b_lo + 6, idesc, 1);
+                const uint32_t sa = base + st * stage_bytes;
+                const uint64_t a0 = desc0 + (sa >> 4), b0 = a0 + static_cast<uint32_t>(p.kg) * (kABytes >> 4);
+                const int g_end = min(p.kg, p.kchunks - kq * p.kg);
+                if (elect_one()) {
+                    for (int g = 0; g < g_end; g++) {
+                        const uint64_t ad = a0 + static_cast<uint32_t>(g) * (kABytes >> 4), bd = b0 + static_cast<uint32_t>(g) * b_chunk16;
+                        const int ksteps = (kq * p.kg + g == p.kchunks - 1) ? p.ksteps_last : 4;
+                        umma_f16(d_tmem, ad, bd, idesc, (ki | g) != 0);
+                        if (ksteps > 1) umma_f16(d_tmem, ad + 2, bd + 2, idesc, 1);
+                        if (ksteps > 2) umma_f16(d_tmem, ad + 4, bd + 4, idesc, 1);
+                        if (ksteps > 3) umma_f16(d_tmem, ad + 6, bd + 6, idesc, 1);
                     }
                     umma_commit(&empty_bar[st]);  // frees the stage once these MMAs have read it
-                    if (++kq == p.kgroups) kq = 0;
                 }
-                if (ok) umma_commit(&tfull_bar[acc]);
-                if (j == 0) DLF_TRACE_POINT(p.status, 4);
+                __syncwarp();
+                if (++kq == p.kgroups) kq = 0;
             }
+            if (ok && elect_one()) umma_commit(&tfull_bar[acc]);
+            __syncwarp();
+            if (j == 0 && lane == 0) DLF_TRACE_POINT(p.status, 4);
         }
     } else {
         // ---- epilogue warps ---------------------------------------------------------------------------

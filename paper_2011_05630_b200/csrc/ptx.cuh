@@ -27,11 +27,14 @@ __device__ __forceinline__ uint64_t global_ns() {
 #define DLF_TRACE_DECL(acc, mark) long long acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}; long long mark = clock64()
 #define DLF_TRACE_ACC(acc, slot, mark) do { const long long now_ = clock64(); acc[slot] += now_ - mark; mark = now_; } while (0)
 #define DLF_TRACE_FLUSH(status, acc) do { if (blockIdx.x == 0 && threadIdx.x == 0) for (int i_ = 0; i_ < 8; i_++) reinterpret_cast<volatile long long*>(status)[4 + i_] = acc[i_]; } while (0)
+// the same for any one thread of CTA 0, into slots base .. base + 7
+#define DLF_TRACE_FLUSH_AT(status, acc, base) do { if (blockIdx.x == 0) for (int i_ = 0; i_ < 8; i_++) reinterpret_cast<volatile long long*>(status)[4 + (base) + i_] = acc[i_]; } while (0)
 #else
 #define DLF_TRACE_POINT(status, slot) do { } while (0)
 #define DLF_TRACE_DECL(acc, mark) do { } while (0)
 #define DLF_TRACE_ACC(acc, slot, mark) do { } while (0)
 #define DLF_TRACE_FLUSH(status, acc) do { } while (0)
+#define DLF_TRACE_FLUSH_AT(status, acc, base) do { } while (0)
 #endif
 
 // ---- programmatic dependent launch -----------------------------------------------------------------
@@ -88,6 +91,25 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             }
         }
     }
+}
+
+// Warp-wide form: every lane polls (a whole warp stays on the issue path so that the addresses it
+// computes are warp-uniform values); the result is voted so that the warp leaves a wait together.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                               int* status, int code) {
+    const bool ok = mbar_wait(bar, parity, abort_flag, status, code);
+    return __all_sync(0xffffffffu, ok);
+}
+
+// True in exactly one lane of a converged warp (the same lane every time).
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .b32 rx;\n\t.reg .pred px;\n\t"
+        "elect.sync rx|px, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, px;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
 }
 
 __device__ __forceinline__ void fence_barrier_init() {
@@ -176,8 +198,14 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64
         ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
-// Lean form for the issue loop (one thread issues every UMMA of a CTA, so its instruction count
-// is what bounds small-N MMAs): the descriptors' upper words are constants, only the 14-bit
+// Measured on B200 (M = 128, K = 16, fp16): an issue loop run by ONE thread (`if (lane == 0)`) spends
+// about 72 cycles per UMMA whatever N is, because every descriptor is a per-thread value that has to
+// be moved into uniform registers; the same loop run by the whole warp with warp-uniform descriptors
+// and the UMMA group under elect_one() reaches the hardware's rates: 48 cycles at N = 64 (operand
+// reads from shared memory), N / 2 cycles from N = 128 up.  Descriptors differ only in the 14-bit
+// start-address field, so stepping one is a 64-bit add of (bytes >> 4).
+//
+// Lean 32-bit form (older issue loops): the descriptors' upper words are constants, only the
 // start-address field of the lower word changes from one MMA to the next.
 constexpr uint32_t kDescHiSw128 = (1024u >> 4) | (1u << 14) | (2u << 29);
 __device__ __forceinline__ uint32_t umma_desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
