@@ -293,6 +293,24 @@ static MbconvArgs mbconv_args(const dlf_net* net, int first, int last, const voi
     return a;
 }
 
+// A fully connected layer is a 1x1 convolution over a 1x1 image whose channels are the flattened
+// input (NHWC order, which is how the map lies in memory): the tensor-core kernel then streams the
+// weight matrix through its TMA ring, one slab of output features per CTA.
+static ConvArgs fc_as_conv_args(const dlf_net* net, int i, const void* in_dev, void* out_dev) {
+    const Layer& l = net->layers[i];
+    ConvArgs a;
+    std::memset(&a, 0, sizeof(a));
+    a.x = l.d.src < 0 ? in_dev : slot(net, l.d.src);
+    a.w = l.w;
+    a.bias = l.bias;
+    a.y = out_dev;
+    a.N = static_cast<int>(l.in[0]); a.H = 1; a.W = 1;
+    a.Cin = l.d.cin; a.Ho = 1; a.Wo = 1; a.Cout = l.d.cout;
+    a.kh = 1; a.kw = 1; a.stride = 1; a.pad = 0; a.groups = 1;
+    a.act = l.d.act; a.pool = 0;
+    return a;
+}
+
 static bool single_kind(const dlf_net* net, int i, Kind* kind) {
     const Layer& l = net->layers[i];
     switch (l.d.op) {
@@ -311,6 +329,10 @@ static bool single_kind(const dlf_net* net, int i, Kind* kind) {
             return true;
         case DLF_FC:
             if (l.d.cin % 8) return false;
+            // the CUDA-core kernel re-reads the weights once per 8 images and keeps few bytes in flight: measured
+            // faster only for small matrices at small batch
+            if (!net->opt_no_tc && l.d.res_src == -2 && (l.in[0] > 8 || l.w_elems * 2 >= (16ll << 20)) &&
+                conv_tc_supported(fc_as_conv_args(net, i, nullptr, nullptr))) { *kind = K_CONV_TC; return true; }
             *kind = K_FC;
             return true;
         case DLF_MAXPOOL:
@@ -361,7 +383,9 @@ static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* 
             return launch_chain_tc(a, g.tiling, g.sms, net->opt_base_offset, status, s);
         }
         case K_MBCONV: return launch_mbconv_tc(mbconv_args(net, g.first, g.last, in_dev, y), g.mb_tiling, g.sms, status, s);
-        case K_CONV_TC: return launch_conv_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
+        case K_CONV_TC:
+            if (z.d.op == DLF_FC) return launch_conv_tc(fc_as_conv_args(net, g.first, in_dev, y), g.sms, status, s);
+            return launch_conv_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
         case K_STEM_TC: return launch_stem_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
         case K_CONV_DIRECT: return launch_conv_direct(conv_args(net, g.first, in_dev, y), g.sms, s);
         case K_DW: return launch_dw3x3(conv_args(net, g.first, in_dev, y), g.sms, s);

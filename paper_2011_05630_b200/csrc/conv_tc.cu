@@ -45,9 +45,10 @@ constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA lim
 struct ConvTcParams {
     int N, Ho, Wo, Cout;
     int kh, kw, stride, pad;
-    int TW, TH, TN, tiles_w, tiles_h, tiles_n;
+    int TW, TH, TN, rows, tiles_w, tiles_h, tiles_n;  // rows = TW * TH * TN <= 128 pixels of a tile
     int BN, n_tiles_n, acc_stride;
     int kchunks, ksteps_last;
+    int a_bytes;               // one 64-channel slab of the tile's pixels in a ring stage: rows rounded up to 8, x 128 bytes
     int kg, kgroups, grouped;  // K chunks per ring stage; stages per tap; 1 = 5-d / 4-d maps (cin % 64 == 0)
     int stages;
     int n_work;
@@ -90,7 +91,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* stage0 = smem_raw + (base - smem_u32(smem_raw));
     float* bias_s = reinterpret_cast<float*>(stage0 + p.bias_off);
-    const int stage_bytes = p.kg * (kABytes + p.BN * 128);
+    const int stage_bytes = p.kg * (p.a_bytes + p.BN * 128);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &abort_s;
 
@@ -140,7 +141,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             auto fetch_residual = [&](int t, uint32_t b) {
                 const TileCoord c = decode_work(p, t);
                 const int planes = planes_of(c);
-                mbar_expect_tx(&sfree_bar[b], static_cast<uint32_t>(planes) * kABytes);
+                mbar_expect_tx(&sfree_bar[b], static_cast<uint32_t>(planes * p.rows) * 128u);
                 for (int pl = 0; pl < planes; pl++)
                     tma_load_4d(stage_out + b * p.out_buf_bytes + pl * kABytes, &tmr, &sfree_bar[b], c.co0 + pl * 64, c.wo0, c.ho0, c.n0);
             };
@@ -171,7 +172,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             const int role = warp - kProdWarp0;
             const bool is_b = role >= 2;
             const uint32_t parity = role & 1;
-            const uint32_t my_bytes = static_cast<uint32_t>(p.kg) * (is_b ? static_cast<uint32_t>(p.BN) * 128u : static_cast<uint32_t>(kABytes));
+            const uint32_t my_bytes = static_cast<uint32_t>(p.kg) * (is_b ? static_cast<uint32_t>(p.BN) : static_cast<uint32_t>(p.rows)) * 128u;
             uint32_t it = 0;
             bool ok = true;
             for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x) {
@@ -189,8 +190,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                         uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
                         mbar_expect_tx(&full_bar[st], my_bytes);
                         if (is_b) {
-                            if (p.grouped) tma_load_4d(sa + p.kg * kABytes, &tmw, &full_bar[st], 0, c.co0, tap, kq * p.kg);
-                            else tma_load_3d(sa + kABytes, &tmw, &full_bar[st], kq * 64, tap, c.co0);
+                            if (p.grouped) tma_load_4d(sa + p.kg * p.a_bytes, &tmw, &full_bar[st], 0, c.co0, tap, kq * p.kg);
+                            else tma_load_3d(sa + p.a_bytes, &tmw, &full_bar[st], kq * 64, tap, c.co0);
                         } else {
                             const int wi = c.wo0 * p.stride - p.pad + s, hi = c.ho0 * p.stride - p.pad + r;
                             if (p.grouped) tma_load_5d(sa, &tmx, &full_bar[st], 0, wi, hi, c.n0, kq * p.kg);
@@ -206,6 +207,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         const uint32_t idesc = umma_idesc_f16(p.BN);
         const uint64_t desc0 = umma_desc_sw128(0, 0);
         const uint32_t b_chunk16 = static_cast<uint32_t>(p.BN) * 8u;  // one 64-channel weight slab, in 16-byte units
+        const uint32_t a_chunk16 = static_cast<uint32_t>(p.rows) * 8u; // one 64-channel slab of the tile's pixels (a box of kg slabs is dense)
         uint32_t it = 0, j = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
@@ -222,11 +224,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 if (it == 0 && lane == 0) DLF_TRACE_POINT(p.status, 3);
                 tc_fence_after_sync();
                 const uint32_t sa = base + st * stage_bytes;
-                const uint64_t a0 = desc0 + (sa >> 4), b0 = a0 + static_cast<uint32_t>(p.kg) * (kABytes >> 4);
+                const uint64_t a0 = desc0 + (sa >> 4), b0 = a0 + static_cast<uint32_t>(p.kg * p.a_bytes >> 4);
                 const int g_end = min(p.kg, p.kchunks - kq * p.kg);
                 if (elect_one()) {
                     for (int g = 0; g < g_end; g++) {
-                        const uint64_t ad = a0 + static_cast<uint32_t>(g) * (kABytes >> 4), bd = b0 + static_cast<uint32_t>(g) * b_chunk16;
+                        const uint64_t ad = a0 + static_cast<uint32_t>(g) * a_chunk16, bd = b0 + static_cast<uint32_t>(g) * b_chunk16;
                         const int ksteps = (kq * p.kg + g == p.kchunks - 1) ? p.ksteps_last : 4;
                         umma_f16(d_tmem, ad, bd, idesc, (ki | g) != 0);
                         if (ksteps > 1) umma_f16(d_tmem, ad + 2, bd + 2, idesc, 1);
@@ -257,7 +259,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             const TileCoord c = decode_work(p, t);
             const uint32_t acc = j & 1u;
             const int n = c.n0 + tn, ho = c.ho0 + th, wo = c.wo0 + tw;
-            const bool valid = n < p.N && ho < p.Ho && wo < p.Wo;
+            const bool valid = m < p.rows && n < p.N && ho < p.Ho && wo < p.Wo;
             const long long pix = (static_cast<long long>(n) * p.Ho + ho) * p.Wo + wo;
             const long long opix = POOL ? (static_cast<long long>(n) * Hp + (ho >> 1)) * Wp + (wo >> 1) : pix;
             const bool writer = valid && (!POOL || (((ho | wo) & 1) == 0 && (ho >> 1) < Hp && (wo >> 1) < Wp));
@@ -376,21 +378,38 @@ struct Tile {
     int tw, th, tn;
 };
 
+// Pixel tile TN x TH x TW of at most 128 output pixels (the UMMA's M): the fewest tiles, then the fewest
+// rows (rows past TN * TH * TW are neither loaded nor stored: an image smaller than a power-of-two tile
+// costs no shared-memory fill), then the widest.  The pooled epilogue reduces 2x2 windows with warp
+// shuffles and keeps power-of-two tiles of 128 pixels.
 Tile pick_tile(int N, int Ho, int Wo, int pool) {
     Tile best{16, 8, 1};
     long long best_tiles = -1;
-    for (int tw = 128; tw >= 2; tw >>= 1) {
-        if (pool && tw > 16) continue;
-        for (int th = 128 / tw; th >= 1; th >>= 1) {
-            if (pool && th < 2) continue;
-            const int tn = 128 / (tw * th);
+    if (pool) {
+        for (int tw = 16; tw >= 2; tw >>= 1)
+            for (int th = 128 / tw; th >= 2; th >>= 1) {
+                const int tn = 128 / (tw * th);
+                const long long tiles = static_cast<long long>((Wo + tw - 1) / tw) * ((Ho + th - 1) / th) * ((N + tn - 1) / tn);
+                if (best_tiles < 0 || tiles < best_tiles) {
+                    best_tiles = tiles;
+                    best = Tile{tw, th, tn};
+                }
+            }
+        return best;
+    }
+    int best_rows = 0;
+    for (int tn = 1; tn <= std::min(N, 128); tn++)
+        for (int th = 1; th <= std::min(Ho, 128 / tn); th++) {
+            const int tw_max = std::min(Wo, 128 / (tn * th));
+            const int tw = (Wo + (Wo + tw_max - 1) / tw_max - 1) / ((Wo + tw_max - 1) / tw_max);  // as many tiles per row, evenly wide
+            const int rows = tn * th * tw;
             const long long tiles = static_cast<long long>((Wo + tw - 1) / tw) * ((Ho + th - 1) / th) * ((N + tn - 1) / tn);
-            if (best_tiles < 0 || tiles < best_tiles) {
+            if (best_tiles < 0 || tiles < best_tiles || (tiles == best_tiles && (rows < best_rows || (rows == best_rows && tw > best.tw)))) {
                 best_tiles = tiles;
+                best_rows = rows;
                 best = Tile{tw, th, tn};
             }
         }
-    }
     return best;
 }
 
@@ -432,6 +451,8 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     p.kh = a.kh; p.kw = a.kw; p.stride = a.stride; p.pad = a.pad;
     const Tile tl = pick_tile(a.N, a.Ho, a.Wo, a.pool);
     p.TW = tl.tw; p.TH = tl.th; p.TN = tl.tn;
+    p.rows = tl.tw * tl.th * tl.tn;
+    p.a_bytes = (p.rows + 7) / 8 * 8 * 128;
     p.tiles_w = (a.Wo + tl.tw - 1) / tl.tw;
     p.tiles_h = (a.Ho + tl.th - 1) / tl.th;
     p.tiles_n = (a.N + tl.tn - 1) / tl.tn;
@@ -465,19 +486,21 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     // Two staging buffers (the stores of one tile drain while the next is written) where the ring keeps
     // three stages, or as many as the tile has loads, beside them; else one.
     for (p.out_bufs = a.pool ? 1 : 2; p.out_bufs >= 1; p.out_bufs--) {
-        const int fixed = p.out_bufs * p.out_buf_bytes + bias_bytes + 1024;
+        // the UMMA always reads 128 rows of a slab: behind a shorter one it reads on into whatever follows (those
+        // accumulator rows are never stored), which must still be this CTA's shared memory
+        const int fixed = p.out_bufs * p.out_buf_bytes + bias_bytes + 1024 + (kABytes - p.a_bytes);
         // K chunks per ring stage: every stage costs the issuing threads a fixed handshake (barrier wait,
         // TMA issue, commit), so a stage carries as many 64-channel chunks as leave room for >= 2 stages
         p.kg = 1;
         if (p.grouped)
-            for (int kg : {4, 2})
-                if (kg <= p.kchunks && 2 * kg * (kABytes + p.BN * 128) <= kMaxSmem - fixed && (kg == 2 || 3 * kg * (kABytes + p.BN * 128) <= kMaxSmem - fixed || a.kh * a.kw * ((p.kchunks + kg - 1) / kg) <= 2)) {
+            for (int kg : {8, 4, 2})
+                if (kg <= p.kchunks && (kg < 8 || p.rows <= 32) && 2 * kg * (p.a_bytes + p.BN * 128) <= kMaxSmem - fixed && (kg == 2 || 3 * kg * (p.a_bytes + p.BN * 128) <= kMaxSmem - fixed || a.kh * a.kw * ((p.kchunks + kg - 1) / kg) <= 2)) {
                     p.kg = kg;
                     break;
                 }
         p.kgroups = (p.kchunks + p.kg - 1) / p.kg;
-        const int stage_bytes = p.kg * (kABytes + p.BN * 128);
-        p.stages = std::min(6, (kMaxSmem - fixed) / stage_bytes);
+        const int stage_bytes = p.kg * (p.a_bytes + p.BN * 128);
+        p.stages = std::min(8, (kMaxSmem - fixed) / stage_bytes);
         const int loads = a.kh * a.kw * p.kgroups;
         p.stages = std::max(1, std::min(p.stages, loads));
         p.stage_out_off = p.stages * stage_bytes;
@@ -548,7 +571,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         }
     }
     const int grid = std::max(1, std::min(sm_count, p.n_work));
-    const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024, 120 * 1024);
+    const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024 + (kABytes - p.a_bytes), 120 * 1024);
     cudaError_t e = launch_kernel(pick_kernel(a.act, a.pool != 0, a.res != nullptr), grid, kThreads, smem, s, tmx, tmw, tmy, tmr, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
