@@ -10,8 +10,10 @@
 // over several warps) issue TMA tiled loads (the tap's shifted, strided
 // window of the NHWC input, zero-filled outside the image = the convolution's padding; and the
 // tap's [C_out][64] weight slab) into a ring of 128-byte-swizzled stages; one thread issues
-// tcgen05.mma (fp16 x fp16 -> fp32) into one of two TMEM accumulators; eight epilogue warps (two
-// per TMEM lane quarter, alternating 32-column chunks) drain the other accumulator: bias (staged
+// tcgen05.mma (fp16 x fp16 -> fp32) into one of two TMEM accumulators; sixteen epilogue warps (four
+// per TMEM lane quarter, interleaved 32-column chunks: with two per quarter the schedulers sat idle on
+// the dependent load / add / pack / store chains, measured 1.8 us per 128 x 256 tile) drain the other
+// accumulator: bias (staged
 // in shared memory), residual, activation, fp16 rounding.  Without pooling the tile is written to
 // a swizzled staging buffer (two of them where the ring leaves room) and a separate warp sends it
 // off with TMA stores (clipped at the tensor's edges), waits until they have read the buffer and hands
@@ -34,10 +36,11 @@ namespace dlf {
 
 namespace {
 
-constexpr int kEpiWarps = 8;
-constexpr int kMmaWarp = kEpiWarps;         // warps 0..7 epilogue (warp & 3 = TMEM lane quarter), 8 UMMA issuer,
-constexpr int kProdWarp0 = kEpiWarps + 1;   // 9..12 producers: A even / A odd / B even / B odd ring stages
-constexpr int kStoreWarp = kProdWarp0 + 4;  // 13: TMA stores of finished tiles, TMA loads of residual tiles
+constexpr int kEpiParts = 4;                // epilogue warps per TMEM lane quarter; each takes every kEpiParts-th 32-column chunk
+constexpr int kEpiWarps = 4 * kEpiParts;
+constexpr int kMmaWarp = kEpiWarps;         // warps 0..15 epilogue (warp & 3 = TMEM lane quarter), then the UMMA issuer,
+constexpr int kProdWarp0 = kEpiWarps + 1;   // four producers: A even / A odd / B even / B odd ring stages,
+constexpr int kStoreWarp = kProdWarp0 + 4;  // and one warp for the TMA stores of finished tiles and the TMA loads of residual tiles
 constexpr int kThreads = 32 * (kEpiWarps + 6);
 constexpr int kABytes = 128 * 128;  // 128 pixels x 64 fp16
 constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
@@ -135,15 +138,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
 
     if (warp == kStoreWarp) {
         // ---- staging buffers out (TMA stores) and residual tiles in (TMA loads) ------------------------
-        if (!POOL && lane == 0) {
+        // One lane per 64-channel plane: a thread's bulk copies run one after the other (about 0.3 us each,
+        // measured), the copies of different lanes side by side.
+        if (!POOL) {
             uint8_t* stage_out = stage0 + p.stage_out_off;
             auto planes_of = [&](const TileCoord& c) { return (min(p.BN, ((p.Cout - c.co0) + 15) & ~15) + 63) >> 6; };
             auto fetch_residual = [&](int t, uint32_t b) {
                 const TileCoord c = decode_work(p, t);
                 const int planes = planes_of(c);
-                mbar_expect_tx(&sfree_bar[b], static_cast<uint32_t>(planes * p.rows) * 128u);
-                for (int pl = 0; pl < planes; pl++)
-                    tma_load_4d(stage_out + b * p.out_buf_bytes + pl * kABytes, &tmr, &sfree_bar[b], c.co0 + pl * 64, c.wo0, c.ho0, c.n0);
+                if (lane == 0) mbar_expect_tx(&sfree_bar[b], static_cast<uint32_t>(planes * p.rows) * 128u);
+                __syncwarp();
+                if (lane < planes)
+                    tma_load_4d(stage_out + b * p.out_buf_bytes + lane * kABytes, &tmr, &sfree_bar[b], c.co0 + lane * 64, c.wo0, c.ho0, c.n0);
             };
             if (RES)
                 for (int jj = 0; jj < p.out_bufs; jj++)
@@ -151,17 +157,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             uint32_t j = 0;
             for (int t = blockIdx.x; t < p.n_work; t += gridDim.x, j++) {
                 const uint32_t b = j % p.out_bufs, ph = (j / p.out_bufs) & 1u;
-                if (!mbar_wait(&sfull_bar[b], ph, abort_flag, p.status, 0x500 | (blockIdx.x << 12))) break;
+                if (!mbar_wait_warp(&sfull_bar[b], ph, abort_flag, p.status, 0x500 | (blockIdx.x << 12))) break;
                 const TileCoord c = decode_work(p, t);
-                const int planes = planes_of(c);
-                for (int pl = 0; pl < planes; pl++)
-                    tma_store_4d(&tmy, stage_out + b * p.out_buf_bytes + pl * kABytes, c.co0 + pl * 64, c.wo0, c.ho0, c.n0);
-                tma_store_commit();
-                tma_store_wait_read();  // the buffer has been read: it may take the next residual / the next tile
+                if (lane < planes_of(c)) {
+                    tma_store_4d(&tmy, stage_out + b * p.out_buf_bytes + lane * kABytes, c.co0 + lane * 64, c.wo0, c.ho0, c.n0);
+                    tma_store_commit();
+                    tma_store_wait_read();  // the plane has been read: it may take the next residual / the next tile
+                }
+                __syncwarp();
                 const int t2 = t + p.out_bufs * static_cast<int>(gridDim.x);
                 if (RES) {
                     if (t2 < p.n_work) fetch_residual(t2, b);
-                } else {
+                } else if (lane == 0) {
                     mbar_arrive(&sfree_bar[b]);
                 }
             }
@@ -247,7 +254,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     } else {
         // ---- epilogue warps ---------------------------------------------------------------------------
         const int q = warp & 3;              // TMEM lane quarter this warp may read
-        const int half = warp >> 2;          // which of the alternating 32-column chunks
+        const int part = warp >> 2;          // which of the interleaved 32-column chunks
         const int m = q * 32 + lane;
         const int tw = m % p.TW, th = (m / p.TW) % p.TH, tn = m / (p.TW * p.TH);
         const int Hp = POOL ? p.Ho / 2 : p.Ho, Wp = POOL ? p.Wo / 2 : p.Wo;
@@ -279,7 +286,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     okm |= (okg ? 1u : 0u) << g;
                 }
             };
-            if (RES && POOL) res_load(half * 32, rcur, rok);
+            if (RES && POOL) res_load(part * 32, rcur, rok);
             uint8_t* sout = stage_out + (j % p.out_bufs) * p.out_buf_bytes;
             if (!POOL) {   // the staging buffer is free (first uses pass at once) / holds this tile's residual
                 const uint32_t ph = (j / p.out_bufs) & 1u;
@@ -291,13 +298,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 5);
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.acc_stride;
-            for (int cc = half * 32; cc < ncols; cc += 64) {
-                float v[32];
-                __syncwarp();  // the aligned TMEM load needs the whole warp converged
+            // One 32-column chunk of the accumulator row: bias, residual, activation, rounding, store.
+            auto drain = [&](const uint32_t (&r)[32], int cc) {
                 const int nc = min(32, ncols - cc);
-                if (RES && POOL && cc + 64 < ncols) res_load(cc + 64, rnext, rok_next);
-                if (nc == 32) tmem_ld32(taddr + cc, v);
-                else tmem_ld16(taddr + cc, v);
+                if (RES && POOL && cc + 32 * kEpiParts < ncols) res_load(cc + 32 * kEpiParts, rnext, rok_next);
 #pragma unroll
                 for (int g = 0; g < 4; g++) {
                     if (g * 8 >= nc) break;
@@ -305,8 +309,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     float a[8];
                     const float4 b0 = *reinterpret_cast<const float4*>(bias_s + co);
                     const float4 b1 = *reinterpret_cast<const float4*>(bias_s + co + 4);
-                    a[0] = v[g * 8 + 0] + b0.x; a[1] = v[g * 8 + 1] + b0.y; a[2] = v[g * 8 + 2] + b0.z; a[3] = v[g * 8 + 3] + b0.w;
-                    a[4] = v[g * 8 + 4] + b1.x; a[5] = v[g * 8 + 5] + b1.y; a[6] = v[g * 8 + 6] + b1.z; a[7] = v[g * 8 + 7] + b1.w;
+                    a[0] = __uint_as_float(r[g * 8 + 0]) + b0.x; a[1] = __uint_as_float(r[g * 8 + 1]) + b0.y; a[2] = __uint_as_float(r[g * 8 + 2]) + b0.z; a[3] = __uint_as_float(r[g * 8 + 3]) + b0.w;
+                    a[4] = __uint_as_float(r[g * 8 + 4]) + b1.x; a[5] = __uint_as_float(r[g * 8 + 5]) + b1.y; a[6] = __uint_as_float(r[g * 8 + 6]) + b1.z; a[7] = __uint_as_float(r[g * 8 + 7]) + b1.w;
                     const int g8 = (cc >> 3) + g;
                     uint4* sptr = reinterpret_cast<uint4*>(sout + (g8 >> 3) * kABytes + m * 128 + (((g8 & 7) ^ (m & 7)) << 4));
                     if (RES && !POOL) {   // the residual tile was loaded into the staging buffer (zero outside the tensor)
@@ -351,6 +355,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     for (int g = 0; g < 4; g++) rcur[g] = rnext[g];
                     rok = rok_next;
                 }
+            };
+            for (int cc = part * 32; cc < ncols; cc += 32 * kEpiParts) {
+                uint32_t r[32];
+                __syncwarp();  // the aligned TMEM load needs the whole warp converged
+                tmem_ld32_issue(taddr + cc, r);
+                tmem_ld32_wait(r);
+                drain(r, cc);
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -457,14 +468,21 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     p.tiles_h = (a.Ho + tl.th - 1) / tl.th;
     p.tiles_n = (a.N + tl.tn - 1) / tl.tn;
     const int cout16 = (a.Cout + 15) / 16 * 16;
-    // Channel tile: layers with few pixel tiles (small images, small batch) get narrower channel tiles so
-    // that the work list covers the SMs; cost = waves x (tile width + a fixed per-item overhead).  With
-    // several channel tiles the width is a multiple of 64, so that a tile's 64-channel TMA store boxes
-    // never reach into its neighbour's channels.
-    {
-        const long long m_tiles = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n;
+    p.kchunks = (a.Cin + 63) / 64;
+    p.ksteps_last = ((a.Cin - (p.kchunks - 1) * 64) + 15) / 16;
+    p.grouped = (a.Cin % 64 == 0) ? 1 : 0;
+    const long long m_tiles = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n;
+    int bias_bytes = 0;
+    // Lays out the ring, the staging buffers and the bias for a shared-memory budget and a widest channel tile;
+    // false if not even a two-stage ring (or all of the tile's loads) fits.
+    auto configure = [&](int budget, int bn_max, int min_stages) {
+        // Channel tile: layers with few pixel tiles (small images, small batch) get narrower channel tiles so
+        // that the work list covers the SMs; cost = waves x (tile width + a fixed per-item overhead).  With
+        // several channel tiles the width is a multiple of 64, so that a tile's 64-channel TMA store boxes
+        // never reach into its neighbour's channels.
         long long best_cost = -1;
         for (int bn : {256, 192, 128, 64}) {
+            if (bn > bn_max) continue;
             const int width = std::min(bn, cout16);
             const int nt = (cout16 + width - 1) / width;
             if (nt > 1 && width % 64) continue;
@@ -476,37 +494,38 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
                 p.n_tiles_n = nt;
             }
         }
-    }
-    p.kchunks = (a.Cin + 63) / 64;
-    p.ksteps_last = ((a.Cin - (p.kchunks - 1) * 64) + 15) / 16;
-    const int out_planes = a.pool ? 0 : (p.BN + 63) / 64;
-    const int bias_bytes = (p.n_tiles_n * p.BN * 4 + 1023) / 1024 * 1024;
-    p.grouped = (a.Cin % 64 == 0) ? 1 : 0;
-    p.out_buf_bytes = out_planes * kABytes;
-    // Two staging buffers (the stores of one tile drain while the next is written) where the ring keeps
-    // three stages, or as many as the tile has loads, beside them; else one.
-    for (p.out_bufs = a.pool ? 1 : 2; p.out_bufs >= 1; p.out_bufs--) {
-        // the UMMA always reads 128 rows of a slab: behind a shorter one it reads on into whatever follows (those
-        // accumulator rows are never stored), which must still be this CTA's shared memory
-        const int fixed = p.out_bufs * p.out_buf_bytes + bias_bytes + 1024 + (kABytes - p.a_bytes);
-        // K chunks per ring stage: every stage costs the issuing threads a fixed handshake (barrier wait,
-        // TMA issue, commit), so a stage carries as many 64-channel chunks as leave room for >= 2 stages
-        p.kg = 1;
-        if (p.grouped)
-            for (int kg : {8, 4, 2})
-                if (kg <= p.kchunks && (kg < 8 || p.rows <= 32) && 2 * kg * (p.a_bytes + p.BN * 128) <= kMaxSmem - fixed && (kg == 2 || 3 * kg * (p.a_bytes + p.BN * 128) <= kMaxSmem - fixed || a.kh * a.kw * ((p.kchunks + kg - 1) / kg) <= 2)) {
-                    p.kg = kg;
-                    break;
-                }
-        p.kgroups = (p.kchunks + p.kg - 1) / p.kg;
-        const int stage_bytes = p.kg * (p.a_bytes + p.BN * 128);
-        p.stages = std::min(8, (kMaxSmem - fixed) / stage_bytes);
-        const int loads = a.kh * a.kw * p.kgroups;
-        p.stages = std::max(1, std::min(p.stages, loads));
-        p.stage_out_off = p.stages * stage_bytes;
-        p.bias_off = p.stage_out_off + p.out_bufs * p.out_buf_bytes;
-        if (p.out_bufs == 1 || p.stages >= std::min(3, loads)) break;
-    }
+        if (best_cost < 0) return false;
+        const int out_planes = a.pool ? 0 : (p.BN + 63) / 64;
+        bias_bytes = (p.n_tiles_n * p.BN * 4 + 1023) / 1024 * 1024;
+        p.out_buf_bytes = out_planes * kABytes;
+        const int loads_min = a.kh * a.kw * p.kchunks;
+        // Two staging buffers (the stores of one tile drain while the next is written) where the ring keeps
+        // three stages, or as many as the tile has loads, beside them; else one.
+        for (p.out_bufs = a.pool ? 1 : 2; p.out_bufs >= 1; p.out_bufs--) {
+            // the UMMA always reads 128 rows of a slab: behind a shorter one it reads on into whatever follows (those
+            // accumulator rows are never stored), which must still be this CTA's shared memory
+            const int fixed = p.out_bufs * p.out_buf_bytes + bias_bytes + 1024 + (kABytes - p.a_bytes);
+            // K chunks per ring stage: every stage costs the issuing threads a fixed handshake (barrier wait,
+            // TMA issue, commit), so a stage carries as many 64-channel chunks as leave room for >= 2 stages
+            p.kg = 1;
+            if (p.grouped)
+                for (int kg : {8, 4, 2})
+                    if (kg <= p.kchunks && (kg < 8 || p.rows <= 32) && 2 * kg * (p.a_bytes + p.BN * 128) <= budget - fixed && (kg == 2 || 3 * kg * (p.a_bytes + p.BN * 128) <= budget - fixed || a.kh * a.kw * ((p.kchunks + kg - 1) / kg) <= 2)) {
+                        p.kg = kg;
+                        break;
+                    }
+            p.kgroups = (p.kchunks + p.kg - 1) / p.kg;
+            const int stage_bytes = p.kg * (p.a_bytes + p.BN * 128);
+            p.stages = std::min(8, (budget - fixed) / stage_bytes);
+            const int loads = a.kh * a.kw * p.kgroups;
+            p.stages = std::min(p.stages, loads);
+            p.stage_out_off = p.stages * stage_bytes;
+            p.bias_off = p.stage_out_off + p.out_bufs * p.out_buf_bytes;
+            if (p.stages >= 1 && (p.out_bufs == 1 || p.stages >= std::min(3, loads))) break;
+        }
+        return p.stages >= std::min(min_stages, loads_min);
+    };
+    if (!configure(kMaxSmem, 256, 1)) return DLF_E_UNSUPPORTED;
     const long long n_work = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n * p.n_tiles_n;
     if (n_work > 0x7fffffffLL) return DLF_E_UNSUPPORTED;
     p.n_work = static_cast<int>(n_work);
@@ -571,6 +590,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         }
     }
     const int grid = std::max(1, std::min(sm_count, p.n_work));
+    // never two of these CTAs on an SM: each may hold all of tensor memory
     const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024 + (kABytes - p.a_bytes), 120 * 1024);
     cudaError_t e = launch_kernel(pick_kernel(a.act, a.pool != 0, a.res != nullptr), grid, kThreads, smem, s, tmx, tmw, tmy, tmr, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
