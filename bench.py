@@ -204,6 +204,28 @@ def group_report(sess, B, xd, flush, stream, pk):
     return rows
 
 
+def layer_report(sess, B, layers, xd, stream, pk, sms):
+    """One row per layer run alone on all SMs: precise device time of one launch (dlf_net_time_span: four
+    back-to-back launches, warm L2) beside the layer's roofline at the measured peaks."""
+    sess.set_plan(None, None)
+    kern = sess.kernels()
+    rows, first = [], True
+    for i, l in enumerate(layers):
+        ms = B.net_time_span(sess.net, i, i, sms, xd.data_ptr(), stream.cuda_stream, 2, 7, prepare=first)
+        first = False
+        fl, by, _, _ = B.net_group_model(sess.net, i)
+        t_fl = fl / (pk["bf16_tflops_sustained"] * 1e12) * 1e3 if kern[i] in ("chain_tc", "conv_tc") else 0.0
+        t_by = by / (pk["hbm_gbs"] * 1e9) * 1e3
+        rows.append((i, kern[i], l["op"], l["cin"], l["cout"], l["kh"], l["stride"], B.net_layer_info(sess.net, i)[2], ms, t_fl, t_by))
+    sys.stderr.write("| # | kernel | layer | out | us | roof us (tensor / HBM) | frac |\n|---|---|---|---|---|---|---|\n")
+    for i, k, op, cin, cout, kh, st, sh, ms, t_fl, t_by in rows:
+        roof = max(t_fl, t_by)
+        sys.stderr.write("| %d | %s | %s %d->%d k%d s%d | %dx%d | %.1f | %.1f (%.1f / %.1f) | %.2f |\n" % (
+            i, k, op, cin, cout, kh, st, sh[1], sh[2], ms * 1e3, roof * 1e3, t_fl * 1e3, t_by * 1e3, roof / ms))
+    tot, roof = sum(r[8] for r in rows), sum(max(r[9], r[10]) for r in rows)
+    sys.stderr.write("sum %.1f us, roofline %.1f us, fraction %.3f\n" % (tot * 1e3, roof * 1e3, roof / tot))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -214,6 +236,7 @@ def main():
     ap.add_argument("--bruteforce", action="store_true", help="also time the reduced brute-force plan")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--groups", action="store_true", help="print the per-group table to stderr")
+    ap.add_argument("--layers", action="store_true", help="print a per-layer table (each layer alone, precise times) to stderr")
     ap.add_argument("--op-critical", type=float, default=None, help="override Algorithm 1's critical operation count per SM")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
@@ -299,6 +322,8 @@ def main():
                 sys.stderr.write("%-12s %3d-%3d sms=%3d %8.4f ms roof %8.4f ms frac %.3f %s red %.2f\n" % (
                     r["k"], r["first"], r["last"], r["sms"], r["ms"], r["t_roof_ms"], r["t_roof_ms"] / max(r["ms"], 1e-9),
                     r["bound"], r["redundancy"]))
+        if args.layers:
+            layer_report(sess, B, layers, xd, stream, pk, sms)
         if args.groups:
             sess.set_plan(None, None)
             show(group_report(sess, B, xd, flush, stream, pk), "unfused")
