@@ -236,6 +236,7 @@ def main():
     ap.add_argument("--bruteforce", action="store_true", help="also time the reduced brute-force plan")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--groups", action="store_true", help="print the per-group table to stderr")
+    ap.add_argument("--ablation", action="store_true", help="also time the strategies of the paper's ablation (Table 3); table to stderr")
     ap.add_argument("--layers", action="store_true", help="print a per-layer table (each layer alone, precise times) to stderr")
     ap.add_argument("--op-critical", type=float, default=None, help="override Algorithm 1's critical operation count per SM")
     args = ap.parse_args()
@@ -297,6 +298,31 @@ def main():
             clocks = sampler.stop()
         value, total_ms = D.job_throughput(sum(ms), batch * args.steps, device=sess.device)
         results[name] = {"ms_per_step": total_ms / args.steps, "n_groups": sess.n_groups, "value": value}
+
+    ablation = None
+    if args.ablation:
+        ablation = []
+        k_steps = max(3, min(args.steps, 20))
+        for name, e, s in plans.ablation_plans(sess.net, len(layers), sms):
+            tries = [s] if s is not None else [[f] * len(e) for f in plans.sm_fractions(sms)]
+            best = None
+            for smc in tries:
+                sess.set_plan(e, smc)
+                barrier()
+                few = 2 if max(smc) == 1 else k_steps   # one SM: a step takes ~150x longer
+                ms = time_plan(sess, B, torch, xd, few, min(args.warmup, 3 if few > 2 else 1), flush, stream)
+                barrier()
+                value, total_ms = D.job_throughput(sum(ms), batch * few, device=sess.device)
+                if best is None or value > best["value"]:
+                    best = {"strategy": name, "ms_per_step": total_ms / few, "n_groups": sess.n_groups, "value": value, "sm_count": max(smc)}
+            ablation.append(best)
+        for r in ablation:
+            r["speedup_over_strategy_1"] = r["value"] / ablation[0]["value"]
+        if rank == 0:
+            sys.stderr.write("---- ablation (paper Table 3) ----\n| strategy | groups | S (max) | ms / step | images/s | x strategy 1 |\n|---|---|---|---|---|---|\n")
+            for r in ablation:
+                sys.stderr.write("| %s | %d | %d | %.4f | %.0f | %.2f |\n" % (r["strategy"], r["n_groups"], r["sm_count"], r["ms_per_step"],
+                                                                            r["value"], r["speedup_over_strategy_1"]))
 
     # end to end through the host-buffer entry point: pinned host input, H2D, run, D2H, per step
     sess.set_plan(t_ends, t_sms)
@@ -365,6 +391,8 @@ def main():
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "clocks": clocks,
                 "gpu_launches": args.steps * tuned["n_groups"],
                 "paper_context": "3.6x-7.9x over no-fusion/MP=1 on a Cambricon MLU100 (other hardware)"}
+        if ablation is not None:
+            line["ablation"] = ablation
         if "bruteforce" in results:
             line["bruteforce"] = results["bruteforce"]
             line["tuned_over_bruteforce"] = tuned["value"] / results["bruteforce"]["value"]

@@ -19,3 +19,22 @@ def tuned_plan(net, n_layers, **over):
 def sm_fractions(sms):
     """The paper's reduced core-count set {1,2,4,8,12,16,24,32}/32 scaled to this device."""
     return sorted({max(1, round(sms * f / 32)) for f in (1, 2, 4, 8, 12, 16, 24, 32)})
+
+
+def ablation_plans(net, n_layers, sms, **over):
+    """The execution strategies of the paper's ablation (Table 3), as (name, group_end, sm_count) with None for
+    "to be searched": 1 no fusion on one SM; 2 no fusion, one network-wide SM count (the caller tries
+    sm_fractions and keeps the best); 3 no fusion, every layer on its own Eq. 5 count; 4 everything fused that
+    can be, all SMs; 5 Algorithm 1's blocks, all SMs; 6 Algorithm 1's blocks and SM counts.  Strategy 3 is
+    Algorithm 1 with a vanishing critical operation count (every layer closes its own block), strategy 4 with an
+    unreachable one (a block closes only where it must)."""
+    every = list(range(n_layers))
+    per_layer = tuned_plan(net, n_layers, **dict(over, op_critical=1e-30))
+    all_fused = tuned_plan(net, n_layers, **dict(over, op_critical=1e300))
+    tuned = tuned_plan(net, n_layers, **over)
+    return [("1 no fusion, 1 SM", every, [1] * n_layers),
+            ("2 no fusion, best fixed S", every, None),
+            ("3 no fusion, per-layer S (Eq. 5)", per_layer[0], per_layer[1]),
+            ("4 all fused, all SMs", all_fused[0], [sms] * len(all_fused[0])),
+            ("5 Algorithm 1 blocks, all SMs", tuned[0], [sms] * len(tuned[0])),
+            ("6 Algorithm 1 blocks and SM counts", tuned[0], tuned[1])]
