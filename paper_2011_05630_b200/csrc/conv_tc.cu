@@ -22,6 +22,11 @@
 // output pixel per thread, direct residual loads would touch 32 cache lines per instruction and
 // were measured to double the time of the memory-bound 1x1 layers.  With the fused 2x2 max-pool
 // the window is reduced by warp shuffles and written with 16-byte stores.
+// Row mode (3x3, stride 1, whole 64-channel chunks, images up to 126 pixels wide): a tile is whole output rows seen
+// with a pitch of W + 2, so the three taps of a kernel row are ONE loaded window read through UMMA descriptors that
+// start 0, 1 and 2 pixels into it; the window crosses L2 -> shared memory three times per chunk instead of nine.
+// Chosen where it cuts the bytes a CTA streams by a fifth or more (measured: 64 -> 128 at 112x112 34 -> 23 us,
+// 512 -> 512 at 14x14 23 -> 17 us, the ResNet-50 3x3 layers 8 % faster; neutral where the weight slabs dominate).
 // The epilogue is specialised at compile time on (activation, pool, residual): it is the part of
 // the kernel that bounds memory-bound layers, and runtime branches there cost more than the math.
 #include <cuda.h>
@@ -52,6 +57,7 @@ struct ConvTcParams {
     int BN, n_tiles_n, acc_stride;
     int kchunks, ksteps_last;
     int a_bytes;               // one 64-channel slab of the tile's pixels in a ring stage: rows rounded up to 8, x 128 bytes
+    int tps, tgroups;          // taps per ring stage (3 = a whole kernel row, see the row mode) and tap groups per K-chunk group
     int kg, kgroups, grouped;  // K chunks per ring stage; stages per tap; 1 = 5-d / 4-d maps (cin % 64 == 0)
     int stages;
     int n_work;
@@ -80,7 +86,7 @@ __device__ __forceinline__ TileCoord decode_work(const ConvTcParams& p, int t) {
     return c;
 }
 
-template <int ACT, bool POOL, bool RES>
+template <int ACT, bool POOL, bool RES, bool ROW>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
                const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmr, const ConvTcParams p) {
@@ -94,7 +100,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* stage0 = smem_raw + (base - smem_u32(smem_raw));
     float* bias_s = reinterpret_cast<float*>(stage0 + p.bias_off);
-    const int stage_bytes = p.kg * (p.a_bytes + p.BN * 128);
+    constexpr int kTps = ROW ? 3 : 1;   // taps per ring stage: a whole kernel row in the row mode
+    const int stage_bytes = p.kg * (p.a_bytes + kTps * p.BN * 128);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &abort_s;
 
@@ -134,7 +141,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
     const int taps = p.kh * p.kw;
-    const int k_iters = taps * p.kgroups;
+    const int k_iters = p.tgroups * p.kgroups;
 
     if (warp == kStoreWarp) {
         // ---- staging buffers out (TMA stores) and residual tiles in (TMA loads) ------------------------
@@ -155,9 +162,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 for (int jj = 0; jj < p.out_bufs; jj++)
                     if (static_cast<int>(blockIdx.x) + jj * static_cast<int>(gridDim.x) < p.n_work) fetch_residual(blockIdx.x + jj * gridDim.x, jj);
             uint32_t j = 0;
+            DLF_TRACE_DECL(sacc, smark);  // cycles of CTA 0's store warp: 0 wait for a staged tile, 1 store and its read, 2 residual fetch
             for (int t = blockIdx.x; t < p.n_work; t += gridDim.x, j++) {
                 const uint32_t b = j % p.out_bufs, ph = (j / p.out_bufs) & 1u;
                 if (!mbar_wait_warp(&sfull_bar[b], ph, abort_flag, p.status, 0x500 | (blockIdx.x << 12))) break;
+                DLF_TRACE_ACC(sacc, 0, smark);
                 const TileCoord c = decode_work(p, t);
                 if (lane < planes_of(c)) {
                     tma_store_4d(&tmy, stage_out + b * p.out_buf_bytes + lane * kABytes, c.co0 + lane * 64, c.wo0, c.ho0, c.n0);
@@ -165,13 +174,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     tma_store_wait_read();  // the plane has been read: it may take the next residual / the next tile
                 }
                 __syncwarp();
+                DLF_TRACE_ACC(sacc, 1, smark);
                 const int t2 = t + p.out_bufs * static_cast<int>(gridDim.x);
                 if (RES) {
                     if (t2 < p.n_work) fetch_residual(t2, b);
                 } else if (lane == 0) {
                     mbar_arrive(&sfree_bar[b]);
                 }
+                DLF_TRACE_ACC(sacc, 2, smark);
             }
+            if (lane == 0) DLF_TRACE_FLUSH_N(p.status, sacc, 11, 3);
         }
     } else if (warp >= kProdWarp0) {
         // ---- producers: TMA loads into the stage ring -------------------------------------------
@@ -179,12 +191,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             const int role = warp - kProdWarp0;
             const bool is_b = role >= 2;
             const uint32_t parity = role & 1;
-            const uint32_t my_bytes = static_cast<uint32_t>(p.kg) * (is_b ? static_cast<uint32_t>(p.BN) : static_cast<uint32_t>(p.rows)) * 128u;
+            const uint32_t my_bytes = static_cast<uint32_t>(p.kg) * (is_b ? static_cast<uint32_t>(kTps * p.BN) : static_cast<uint32_t>(p.rows)) * 128u;
             uint32_t it = 0;
             bool ok = true;
+            DLF_TRACE_DECL(pacc, pmark);  // cycles of CTA 0's producers: 0 wait for a free stage, 1 issue
             for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x) {
                 const TileCoord c = decode_work(p, t);
-                for (int tap = 0; tap < taps && ok; tap++) {
+                for (int tg = 0; tg < p.tgroups && ok; tg++) {
+                    // row mode: tap group tg = kernel row tg, its window loaded once at the row's first tap
+                    const int tap = tg * kTps;
                     const int r = tap / p.kw, s = tap % p.kw;
                     for (int kq = 0; kq < p.kgroups; kq++, it++) {
                         const int st = it % p.stages;
@@ -194,6 +209,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                         ok = mbar_wait(&empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status,
                                        0x100 | (blockIdx.x << 12));
                         if (!ok) break;
+                        DLF_TRACE_ACC(pacc, 0, pmark);
                         uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
                         mbar_expect_tx(&full_bar[st], my_bytes);
                         if (is_b) {
@@ -205,9 +221,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                             else tma_load_4d(sa, &tmx, &full_bar[st], kq * 64, wi, hi, c.n0);
                         }
                         if (it == 0) DLF_TRACE_POINT(p.status, 2);
+                        DLF_TRACE_ACC(pacc, 1, pmark);
                     }
                 }
             }
+            DLF_TRACE_FLUSH_N(p.status, pacc, 17 + 2 * role, 2);
         }
     } else if (warp == kMmaWarp) {
         // ---- MMA issuer: the whole warp walks the loop (warp-uniform addresses), one elected lane issues ----
@@ -217,10 +235,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         const uint32_t a_chunk16 = static_cast<uint32_t>(p.rows) * 8u; // one 64-channel slab of the tile's pixels (a box of kg slabs is dense)
         uint32_t it = 0, j = 0;
         bool ok = true;
+        DLF_TRACE_DECL(macc, mmark);  // cycles of CTA 0's issuer: 0 accumulator wait, 1 stage wait, 2 issue
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
             const uint32_t acc = j & 1u;
             ok = mbar_wait_warp(&tempty_bar[acc], ((j >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x200 | (blockIdx.x << 12));
             if (!ok) break;
+            DLF_TRACE_ACC(macc, 0, mmark);
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + acc * p.acc_stride;
             int kq = 0;
@@ -229,28 +249,46 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 ok = mbar_wait_warp(&full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                 if (!ok) break;
                 if (it == 0 && lane == 0) DLF_TRACE_POINT(p.status, 3);
+                DLF_TRACE_ACC(macc, 1, mmark);
                 tc_fence_after_sync();
                 const uint32_t sa = base + st * stage_bytes;
                 const uint64_t a0 = desc0 + (sa >> 4), b0 = a0 + static_cast<uint32_t>(p.kg * p.a_bytes >> 4);
                 const int g_end = min(p.kg, p.kchunks - kq * p.kg);
                 if (elect_one()) {
-                    for (int g = 0; g < g_end; g++) {
-                        const uint64_t ad = a0 + static_cast<uint32_t>(g) * a_chunk16, bd = b0 + static_cast<uint32_t>(g) * b_chunk16;
-                        const int ksteps = (kq * p.kg + g == p.kchunks - 1) ? p.ksteps_last : 4;
-                        umma_f16(d_tmem, ad, bd, idesc, (ki | g) != 0);
-                        if (ksteps > 1) umma_f16(d_tmem, ad + 2, bd + 2, idesc, 1);
-                        if (ksteps > 2) umma_f16(d_tmem, ad + 4, bd + 4, idesc, 1);
-                        if (ksteps > 3) umma_f16(d_tmem, ad + 6, bd + 6, idesc, 1);
+                    if (!ROW) {
+                        for (int g = 0; g < g_end; g++) {
+                            const uint64_t ad = a0 + static_cast<uint32_t>(g) * a_chunk16, bd = b0 + static_cast<uint32_t>(g) * b_chunk16;
+                            const int ksteps = (kq * p.kg + g == p.kchunks - 1) ? p.ksteps_last : 4;
+                            umma_f16(d_tmem, ad, bd, idesc, (ki | g) != 0);
+                            if (ksteps > 1) umma_f16(d_tmem, ad + 2, bd + 2, idesc, 1);
+                            if (ksteps > 2) umma_f16(d_tmem, ad + 4, bd + 4, idesc, 1);
+                            if (ksteps > 3) umma_f16(d_tmem, ad + 6, bd + 6, idesc, 1);
+                        }
+                    } else {
+                        // row mode (whole 64-channel chunks): the three taps of a kernel row read the same window, one
+                        // pixel (one 128-byte row) further each
+                        for (int g = 0; g < g_end; g++) {
+                            uint64_t ad = a0 + static_cast<uint32_t>(g) * a_chunk16, bd = b0 + static_cast<uint32_t>(g * 3) * b_chunk16;
+#pragma unroll
+                            for (int sx = 0; sx < 3; sx++, ad += 8, bd += b_chunk16) {
+                                umma_f16(d_tmem, ad, bd, idesc, (ki | g | sx) != 0);
+                                umma_f16(d_tmem, ad + 2, bd + 2, idesc, 1);
+                                umma_f16(d_tmem, ad + 4, bd + 4, idesc, 1);
+                                umma_f16(d_tmem, ad + 6, bd + 6, idesc, 1);
+                            }
+                        }
                     }
                     umma_commit(&empty_bar[st]);  // frees the stage once these MMAs have read it
                 }
                 __syncwarp();
+                DLF_TRACE_ACC(macc, 2, mmark);
                 if (++kq == p.kgroups) kq = 0;
             }
             if (ok && elect_one()) umma_commit(&tfull_bar[acc]);
             __syncwarp();
             if (j == 0 && lane == 0) DLF_TRACE_POINT(p.status, 4);
         }
+        if (lane == 0) DLF_TRACE_FLUSH_N(p.status, macc, 14, 3);
     } else {
         // ---- epilogue warps ---------------------------------------------------------------------------
         const int q = warp & 3;              // TMEM lane quarter this warp may read
@@ -262,6 +300,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         const bool issuer = (threadIdx.x == 0);
         uint32_t j = 0;
         bool ok = true;
+        DLF_TRACE_DECL(eacc, emark);  // cycles of CTA 0's first epilogue thread: 0 staging-buffer wait, 1 accumulator wait, 2 drain
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
             const TileCoord c = decode_work(p, t);
             const uint32_t acc = j & 1u;
@@ -293,8 +332,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 ok = mbar_wait(&sfree_bar[j % p.out_bufs], RES ? ph : ph ^ 1u, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
                 if (!ok) break;
             }
+            DLF_TRACE_ACC(eacc, 0, emark);
             ok = mbar_wait(&tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
             if (!ok) break;
+            DLF_TRACE_ACC(eacc, 1, emark);
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 5);
             tc_fence_after_sync();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.acc_stride;
@@ -372,7 +413,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 if (lane == 0) mbar_arrive(&sfull_bar[j % p.out_bufs]);
             }
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 6);
+            DLF_TRACE_ACC(eacc, 2, emark);
         }
+        if (issuer) DLF_TRACE_FLUSH_N(p.status, eacc, 8, 3);
     }
 
     tc_fence_before_sync();
@@ -426,18 +469,23 @@ Tile pick_tile(int N, int Ho, int Wo, int pool) {
 
 typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const ConvTcParams);
 
+template <int ACT, bool POOL, bool RES>
+KernelFn pick_row(bool row) {
+    if constexpr (POOL) return conv_tc_kernel<ACT, POOL, RES, false>;   // the row mode has no pooled epilogue
+    else return row ? conv_tc_kernel<ACT, POOL, RES, true> : conv_tc_kernel<ACT, POOL, RES, false>;
+}
 template <int ACT, bool POOL>
-KernelFn pick_res(bool res) {
-    return res ? conv_tc_kernel<ACT, POOL, true> : conv_tc_kernel<ACT, POOL, false>;
+KernelFn pick_res(bool res, bool row) {
+    return res ? pick_row<ACT, POOL, true>(row) : pick_row<ACT, POOL, false>(row);
 }
 template <int ACT>
-KernelFn pick_pool(bool pool, bool res) {
-    return pool ? pick_res<ACT, true>(res) : pick_res<ACT, false>(res);
+KernelFn pick_pool(bool pool, bool res, bool row) {
+    return pool ? pick_res<ACT, true>(res, row) : pick_res<ACT, false>(res, row);
 }
-KernelFn pick_kernel(int act, bool pool, bool res) {
-    if (act == 0) return pick_pool<0>(pool, res);
-    if (act == 1) return pick_pool<1>(pool, res);
-    return pick_pool<2>(pool, res);
+KernelFn pick_kernel(int act, bool pool, bool res, bool row) {
+    if (act == 0) return pick_pool<0>(pool, res, row);
+    if (act == 1) return pick_pool<1>(pool, res, row);
+    return pick_pool<2>(pool, res, row);
 }
 
 }  // namespace
@@ -460,21 +508,27 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     ConvTcParams p{};
     p.N = a.N; p.Ho = a.Ho; p.Wo = a.Wo; p.Cout = a.Cout;
     p.kh = a.kh; p.kw = a.kw; p.stride = a.stride; p.pad = a.pad;
-    const Tile tl = pick_tile(a.N, a.Ho, a.Wo, a.pool);
-    p.TW = tl.tw; p.TH = tl.th; p.TN = tl.tn;
-    p.rows = tl.tw * tl.th * tl.tn;
-    p.a_bytes = (p.rows + 7) / 8 * 8 * 128;
-    p.tiles_w = (a.Wo + tl.tw - 1) / tl.tw;
-    p.tiles_h = (a.Ho + tl.th - 1) / tl.th;
-    p.tiles_n = (a.N + tl.tn - 1) / tl.tn;
     const int cout16 = (a.Cout + 15) / 16 * 16;
     p.kchunks = (a.Cin + 63) / 64;
     p.ksteps_last = ((a.Cin - (p.kchunks - 1) * 64) + 15) / 16;
     p.grouped = (a.Cin % 64 == 0) ? 1 : 0;
-    const long long m_tiles = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n;
+    Tile tl{};
+    long long m_tiles = 0;
     int bias_bytes = 0;
+    auto set_tile = [&](const Tile& t, int taps_per_stage) {
+        tl = t;
+        p.TW = tl.tw; p.TH = tl.th; p.TN = tl.tn;
+        p.rows = tl.tw * tl.th * tl.tn;
+        p.a_bytes = (p.rows + 7) / 8 * 8 * 128;
+        p.tiles_w = (a.Wo + tl.tw - 1) / tl.tw;
+        p.tiles_h = (a.Ho + tl.th - 1) / tl.th;
+        p.tiles_n = (a.N + tl.tn - 1) / tl.tn;
+        p.tps = taps_per_stage;
+        p.tgroups = a.kh * a.kw / taps_per_stage;
+        m_tiles = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n;
+    };
     // Lays out the ring, the staging buffers and the bias for a shared-memory budget and a widest channel tile;
-    // false if not even a two-stage ring (or all of the tile's loads) fits.
+    // false if not even `min_stages` ring stages (or all of the tile's loads) fit.
     auto configure = [&](int budget, int bn_max, int min_stages) {
         // Channel tile: layers with few pixel tiles (small images, small batch) get narrower channel tiles so
         // that the work list covers the SMs; cost = waves x (tile width + a fixed per-item overhead).  With
@@ -498,26 +552,28 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         const int out_planes = a.pool ? 0 : (p.BN + 63) / 64;
         bias_bytes = (p.n_tiles_n * p.BN * 4 + 1023) / 1024 * 1024;
         p.out_buf_bytes = out_planes * kABytes;
-        const int loads_min = a.kh * a.kw * p.kchunks;
+        const int b_bytes = p.tps * p.BN * 128;   // the weight slabs of one 64-channel chunk in a stage
+        const int loads_min = p.tgroups * p.kchunks;
         // Two staging buffers (the stores of one tile drain while the next is written) where the ring keeps
         // three stages, or as many as the tile has loads, beside them; else one.
         for (p.out_bufs = a.pool ? 1 : 2; p.out_bufs >= 1; p.out_bufs--) {
-            // the UMMA always reads 128 rows of a slab: behind a shorter one it reads on into whatever follows (those
-            // accumulator rows are never stored), which must still be this CTA's shared memory
-            const int fixed = p.out_bufs * p.out_buf_bytes + bias_bytes + 1024 + (kABytes - p.a_bytes);
+            // the UMMA always reads 128 rows of a slab (two more in the row mode): behind a shorter one it reads on
+            // into whatever follows (those accumulator rows are never stored), which must still be this CTA's
+            // shared memory
+            const int fixed = p.out_bufs * p.out_buf_bytes + bias_bytes + 1024 + (kABytes + 256 - p.a_bytes);
             // K chunks per ring stage: every stage costs the issuing threads a fixed handshake (barrier wait,
             // TMA issue, commit), so a stage carries as many 64-channel chunks as leave room for >= 2 stages
             p.kg = 1;
             if (p.grouped)
                 for (int kg : {8, 4, 2})
-                    if (kg <= p.kchunks && (kg < 8 || p.rows <= 32) && 2 * kg * (p.a_bytes + p.BN * 128) <= budget - fixed && (kg == 2 || 3 * kg * (p.a_bytes + p.BN * 128) <= budget - fixed || a.kh * a.kw * ((p.kchunks + kg - 1) / kg) <= 2)) {
+                    if (kg <= p.kchunks && (kg < 8 || p.rows <= 32) && 2 * kg * (p.a_bytes + b_bytes) <= budget - fixed && (kg == 2 || 3 * kg * (p.a_bytes + b_bytes) <= budget - fixed || p.tgroups * ((p.kchunks + kg - 1) / kg) <= 2)) {
                         p.kg = kg;
                         break;
                     }
             p.kgroups = (p.kchunks + p.kg - 1) / p.kg;
-            const int stage_bytes = p.kg * (p.a_bytes + p.BN * 128);
+            const int stage_bytes = p.kg * (p.a_bytes + b_bytes);
             p.stages = std::min(8, (budget - fixed) / stage_bytes);
-            const int loads = a.kh * a.kw * p.kgroups;
+            const int loads = p.tgroups * p.kgroups;
             p.stages = std::min(p.stages, loads);
             p.stage_out_off = p.stages * stage_bytes;
             p.bias_off = p.stage_out_off + p.out_bufs * p.out_buf_bytes;
@@ -525,7 +581,34 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         }
         return p.stages >= std::min(min_stages, loads_min);
     };
+    // What a CTA streams from L2 into shared memory over the kernel (the bound of the 3x3 layers): waves x bytes per item.
+    auto stream_cost = [&]() {
+        const long long waves = (m_tiles * p.n_tiles_n + sm_count - 1) / sm_count;
+        return static_cast<double>(waves) * p.tgroups * p.kchunks * (p.a_bytes + p.tps * p.BN * 128);
+    };
+    // Row mode (3x3, stride 1, pad 1): a tile is TH whole output rows seen with a pitch of Wo + 2, pixel-linear like
+    // its input window, so that the three taps of a kernel row read ONE loaded window through descriptors that
+    // start 0, 1 and 2 pixels (128-byte rows) into it: the window is streamed 3 times per 64-channel chunk instead of
+    // 9 and a stage carries a kernel row's three weight slabs.  The two columns past the image come out as garbage
+    // that the epilogue masks and the clipped TMA store never writes.
+    bool row_mode = false;
+    ConvTcParams p_row{};
+    Tile tl_row{};
+    int bias_row = 0;
+    double cost_row = 0.0;
+    if (a.kh == 3 && a.kw == 3 && a.stride == 1 && a.pad == 1 && !a.pool && p.grouped && a.Wo + 2 <= 128 && a.W == a.Wo && a.H == a.Ho) {
+        set_tile(Tile{a.Wo + 2, std::min(a.Ho, 128 / (a.Wo + 2)), 1}, 3);
+        if (configure(kMaxSmem, 128, 2)) {
+            row_mode = true;
+            p_row = p; tl_row = tl; bias_row = bias_bytes; cost_row = stream_cost();
+        }
+    }
+    set_tile(pick_tile(a.N, a.Ho, a.Wo, a.pool), 1);
     if (!configure(kMaxSmem, 256, 1)) return DLF_E_UNSUPPORTED;
+    if (row_mode && cost_row < 0.8 * stream_cost()) {
+        const long long keep_m = static_cast<long long>(p_row.tiles_w) * p_row.tiles_h * p_row.tiles_n;
+        p = p_row; tl = tl_row; bias_bytes = bias_row; m_tiles = keep_m;
+    }
     const long long n_work = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n * p.n_tiles_n;
     if (n_work > 0x7fffffffLL) return DLF_E_UNSUPPORTED;
     p.n_work = static_cast<int>(n_work);
@@ -552,7 +635,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
         // weights [cout][tap][cin] seen as (64 channels, cout, tap, C_in / 64)
         const uint64_t wdims[4] = {64, static_cast<uint64_t>(a.Cout), taps64, static_cast<uint64_t>(a.Cin / 64)};
         const uint64_t wstrides[3] = {taps64 * a.Cin * 2, static_cast<uint64_t>(a.Cin) * 2, 128};
-        const uint32_t wbox[4] = {64, static_cast<uint32_t>(p.BN), 1, static_cast<uint32_t>(p.kg)};
+        const uint32_t wbox[4] = {64, static_cast<uint32_t>(p.BN), static_cast<uint32_t>(p.tps), static_cast<uint32_t>(p.kg)};
         const uint32_t wes[4] = {1, 1, 1, 1};
         rc = encode_tmap(&tmw, a.w, 4, wdims, wstrides, wbox, wes);
         if (rc) return rc;
@@ -591,8 +674,8 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     }
     const int grid = std::max(1, std::min(sm_count, p.n_work));
     // never two of these CTAs on an SM: each may hold all of tensor memory
-    const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024 + (kABytes - p.a_bytes), 120 * 1024);
-    cudaError_t e = launch_kernel(pick_kernel(a.act, a.pool != 0, a.res != nullptr), grid, kThreads, smem, s, tmx, tmw, tmy, tmr, p);
+    const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024 + (kABytes + 256 - p.a_bytes), 120 * 1024);
+    cudaError_t e = launch_kernel(pick_kernel(a.act, a.pool != 0, a.res != nullptr, p.tps == 3), grid, kThreads, smem, s, tmx, tmw, tmy, tmr, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 
@@ -601,11 +684,12 @@ int conv_tc_init() {
     if (!attr_set) {
         for (int act = 0; act < 3; act++)
             for (int pool = 0; pool < 2; pool++)
-                for (int res = 0; res < 2; res++) {
-                    cudaError_t e = cudaFuncSetAttribute(pick_kernel(act, pool != 0, res != 0),
-                                                         cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-                    if (e != cudaSuccess) return cuda_fail(e);
-                }
+                for (int res = 0; res < 2; res++)
+                    for (int row = 0; row < (pool ? 1 : 2); row++) {
+                        cudaError_t e = cudaFuncSetAttribute(pick_kernel(act, pool != 0, res != 0, row != 0),
+                                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+                        if (e != cudaSuccess) return cuda_fail(e);
+                    }
         attr_set = true;
     }
     return DLF_OK;

@@ -29,12 +29,15 @@ __device__ __forceinline__ uint64_t global_ns() {
 #define DLF_TRACE_FLUSH(status, acc) do { if (blockIdx.x == 0 && threadIdx.x == 0) for (int i_ = 0; i_ < 8; i_++) reinterpret_cast<volatile long long*>(status)[4 + i_] = acc[i_]; } while (0)
 // the same for any one thread of CTA 0, into slots base .. base + 7
 #define DLF_TRACE_FLUSH_AT(status, acc, base) do { if (blockIdx.x == 0) for (int i_ = 0; i_ < 8; i_++) reinterpret_cast<volatile long long*>(status)[4 + (base) + i_] = acc[i_]; } while (0)
+// ... the first n accounts only (the status block holds 28 slots)
+#define DLF_TRACE_FLUSH_N(status, acc, base, n) do { if (blockIdx.x == 0) for (int i_ = 0; i_ < (n); i_++) reinterpret_cast<volatile long long*>(status)[4 + (base) + i_] = acc[i_]; } while (0)
 #else
 #define DLF_TRACE_POINT(status, slot) do { } while (0)
 #define DLF_TRACE_DECL(acc, mark) do { } while (0)
 #define DLF_TRACE_ACC(acc, slot, mark) do { } while (0)
 #define DLF_TRACE_FLUSH(status, acc) do { } while (0)
 #define DLF_TRACE_FLUSH_AT(status, acc, base) do { } while (0)
+#define DLF_TRACE_FLUSH_N(status, acc, base, n) do { } while (0)
 #endif
 
 // ---- programmatic dependent launch -----------------------------------------------------------------
