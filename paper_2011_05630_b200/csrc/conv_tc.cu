@@ -597,7 +597,11 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     int bias_row = 0;
     double cost_row = 0.0;
     if (a.kh == 3 && a.kw == 3 && a.stride == 1 && a.pad == 1 && !a.pool && p.grouped && a.Wo + 2 <= 128 && a.W == a.Wo && a.H == a.Ho) {
-        set_tile(Tile{a.Wo + 2, std::min(a.Ho, 128 / (a.Wo + 2)), 1}, 3);
+        const int th_row = std::min(a.Ho, 128 / (a.Wo + 2));
+        // several whole images per tile where they fit (an image's rows stay together, so the shifted reads of its
+        // valid pixels never reach the next image)
+        const int tn_row = th_row == a.Ho ? std::max(1, std::min(a.N, 128 / (th_row * (a.Wo + 2)))) : 1;
+        set_tile(Tile{a.Wo + 2, th_row, tn_row}, 3);
         if (configure(kMaxSmem, 128, 2)) {
             row_mode = true;
             p_row = p; tl_row = tl; bias_row = bias_bytes; cost_row = stream_cost();
