@@ -19,7 +19,8 @@
 // rounded to fp16 exactly where the layer-by-layer execution rounds it.  Without an expansion layer
 // (the network's first block) steps 1-2 are skipped and the depthwise layer reads the input frame.
 //
-// Warps: 0-7 work (epilogues and depthwise), 8 UMMA issuer, 9 input producer, 10-11 weight producers.
+// Warps: 0-15 work (epilogues and depthwise; a thread keeps FOUR channels' depthwise weights in registers so that
+// sixteen warps fit the register file), 16 UMMA issuer, 17 input producer, 18-19 weight producers.
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -33,7 +34,7 @@ namespace dlf {
 
 namespace {
 
-constexpr int kWorkWarps = 8;
+constexpr int kWorkWarps = 16;   // with eight the CUDA-core phases ran at 0.4 instructions per scheduler cycle (measured)
 constexpr int kMmaWarp = kWorkWarps;
 constexpr int kInWarp = kWorkWarps + 1;
 constexpr int kW1Warp = kWorkWarps + 2;
@@ -65,38 +66,34 @@ __device__ __forceinline__ void work_bar_sync() { asm volatile("bar.sync 1, %0;"
 
 __device__ __forceinline__ float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi); }
 
-// Depthwise 3x3 of one 8-channel group for two horizontally adjacent output pixels: the input
-// vectors the two windows share are read from shared memory and converted once.
+// Depthwise 3x3 of one 4-channel group (8 bytes of a pixel's 128-byte row; g4 = 0..15) for two horizontally
+// adjacent output pixels: the input vectors the two windows share are read from shared memory and converted once.
 template <int STRIDE>
-__device__ __forceinline__ void dw_pair(const uint8_t* hsrc, uint8_t* hdbuf, int fw, int tw, int g8, int oy, int ox, bool second,
-                                        const float (&wreg)[9][8], const float (&breg)[8], float lo, float hi) {
+__device__ __forceinline__ void dw_pair(const uint8_t* hsrc, uint8_t* hdbuf, int fw, int tw, int g4, int oy, int ox, bool second,
+                                        const float (&wreg)[9][4], const float (&breg)[4], float lo, float hi) {
     constexpr int kCols = STRIDE + 3;  // input columns the two windows cover
-    float acc[2][8];
+    const int g8 = g4 >> 1, sub = (g4 & 1) * 8;
+    float acc[2][4];
 #pragma unroll
-    for (int e = 0; e < 8; e++) acc[0][e] = acc[1][e] = 0.0f;
+    for (int e = 0; e < 4; e++) acc[0][e] = acc[1][e] = 0.0f;
 #pragma unroll
     for (int r = 0; r < 3; r++) {
         const int q0 = (oy * STRIDE + r) * fw + ox * STRIDE;
-        uint4 xv[kCols];
+        uint2 xv[kCols];
 #pragma unroll
-        for (int c = 0; c < kCols; c++) xv[c] = *reinterpret_cast<const uint4*>(hsrc + (q0 + c) * 128 + ((g8 ^ ((q0 + c) & 7)) << 4));
+        for (int c = 0; c < kCols; c++) xv[c] = *reinterpret_cast<const uint2*>(hsrc + (q0 + c) * 128 + ((g8 ^ ((q0 + c) & 7)) << 4) + sub);
 #pragma unroll
         for (int c = 0; c < kCols; c++) {
             const __half2* xh = reinterpret_cast<const __half2*>(&xv[c]);
-            float xf[8];
-#pragma unroll
-            for (int e = 0; e < 4; e++) {
-                const float2 f = __half22float2(xh[e]);
-                xf[2 * e] = f.x;
-                xf[2 * e + 1] = f.y;
-            }
+            const float2 f0 = __half22float2(xh[0]), f1 = __half22float2(xh[1]);
+            const float xf[4] = {f0.x, f0.y, f1.x, f1.y};
             if (c < 3) {
 #pragma unroll
-                for (int e = 0; e < 8; e++) acc[0][e] = fmaf(xf[e], wreg[r * 3 + c][e], acc[0][e]);
+                for (int e = 0; e < 4; e++) acc[0][e] = fmaf(xf[e], wreg[r * 3 + c][e], acc[0][e]);
             }
             if (c >= STRIDE) {
 #pragma unroll
-                for (int e = 0; e < 8; e++) acc[1][e] = fmaf(xf[e], wreg[r * 3 + c - STRIDE][e], acc[1][e]);
+                for (int e = 0; e < 4; e++) acc[1][e] = fmaf(xf[e], wreg[r * 3 + c - STRIDE][e], acc[1][e]);
             }
         }
     }
@@ -104,12 +101,10 @@ __device__ __forceinline__ void dw_pair(const uint8_t* hsrc, uint8_t* hdbuf, int
     for (int k = 0; k < 2; k++) {
         if (k == 1 && !second) break;
         const int o = oy * tw + ox + k;
-        uint4 val;
+        uint2 val;
         val.x = pack_half2(clampf(acc[k][0] + breg[0], lo, hi), clampf(acc[k][1] + breg[1], lo, hi));
         val.y = pack_half2(clampf(acc[k][2] + breg[2], lo, hi), clampf(acc[k][3] + breg[3], lo, hi));
-        val.z = pack_half2(clampf(acc[k][4] + breg[4], lo, hi), clampf(acc[k][5] + breg[5], lo, hi));
-        val.w = pack_half2(clampf(acc[k][6] + breg[6], lo, hi), clampf(acc[k][7] + breg[7], lo, hi));
-        *reinterpret_cast<uint4*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4)) = val;
+        *reinterpret_cast<uint2*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4) + sub) = val;
     }
 }
 
@@ -299,7 +294,7 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
     } else {
         // ---- work warps: epilogue 1, depthwise, epilogue 2 ---------------------------------------------------
         const int wt = threadIdx.x;  // 0..255
-        const int q = warp & 3, half = warp >> 2;
+        const int q = warp & 3, part = warp >> 2;   // TMEM lane quarter; which 16-column slice of every 64 columns
         const float lo1 = p.act1 >= 1 ? 0.0f : -INFINITY, hi1 = p.act1 == 2 ? 6.0f : INFINITY;
         const float lo2 = p.act2 >= 1 ? 0.0f : -INFINITY, hi2 = p.act2 == 2 ? 6.0f : INFINITY;
         const float lo3 = p.act3 >= 1 ? 0.0f : -INFINITY, hi3 = p.act3 == 2 ? 6.0f : INFINITY;
@@ -316,26 +311,26 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                 if (!ok) break;
             }
             for (int hc = 0; hc < p.chunks && ok; hc++, cc++) {
-                // this thread's depthwise weights and bias: it keeps one 8-channel group of the chunk for all
-                // its pixels (256 threads, 8 groups: the group index is the thread index modulo 8)
-                const int groups = min(8, (p.hid - hc * 64 + 7) >> 3);  // channel groups this chunk really has
-                float wreg[9][8], breg[8];
+                // this thread's depthwise weights and bias: it keeps one 4-channel group of the chunk for all
+                // its pixels (512 threads, 16 groups: the group index is the thread index modulo 16)
+                const int groups = min(16, (p.hid - hc * 64 + 3) >> 2);  // 4-channel groups this chunk really has
+                float wreg[9][4], breg[4];
                 {
-                    const int ch0 = hc * 64 + (wt & 7) * 8;
-                    if ((wt & 7) < groups) {
-                        __align__(16) __half wv[72];
-                        const uint4* wp4 = reinterpret_cast<const uint4*>(p.wd + static_cast<long long>(ch0) * 9);
+                    const int ch0 = hc * 64 + (wt & 15) * 4;
+                    if ((wt & 15) < groups) {
+                        __align__(8) __half wv[36];   // 4 channels x 9 taps, consecutive in memory from ch0 * 9
+                        const uint2* wp2 = reinterpret_cast<const uint2*>(p.wd + static_cast<long long>(ch0) * 9);
 #pragma unroll
-                        for (int k = 0; k < 9; k++) reinterpret_cast<uint4*>(wv)[k] = __ldg(wp4 + k);
+                        for (int k = 0; k < 9; k++) reinterpret_cast<uint2*>(wv)[k] = __ldg(wp2 + k);
 #pragma unroll
-                        for (int e = 0; e < 8; e++) {
+                        for (int e = 0; e < 4; e++) {
                             breg[e] = __ldg(p.bd + ch0 + e);
 #pragma unroll
                             for (int tp = 0; tp < 9; tp++) wreg[tp][e] = __half2float(wv[e * 9 + tp]);
                         }
                     } else {
 #pragma unroll
-                        for (int e = 0; e < 8; e++) {
+                        for (int e = 0; e < 4; e++) {
                             breg[e] = 0.0f;
 #pragma unroll
                             for (int tp = 0; tp < 9; tp++) wreg[tp][e] = 0.0f;
@@ -352,13 +347,13 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                         const int fy = r / p.fw, fx = r - fy * p.fw;
                         const int gy = iy0 + fy, gx = ix0 + fx;
                         const bool in_img = r < p.FR && gy >= 0 && gy < p.H && gx >= 0 && gx < p.W;
-                        float v[32];
+                        float v[16];
                         __syncwarp();
-                        tmem_ld32(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 64u + half * 32u, v);
+                        tmem_ld16(tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 64u + part * 16u, v);
                         if (r < p.FR) {
-                            const float* bb = bias_s + hc * 64 + half * 32;
+                            const float* bb = bias_s + hc * 64 + part * 16;
 #pragma unroll
-                            for (int g = 0; g < 4; g++) {
+                            for (int g = 0; g < 2; g++) {
                                 uint4 val = make_uint4(0u, 0u, 0u, 0u);
                                 if (in_img) {
                                     const float4 ba = *reinterpret_cast<const float4*>(bb + g * 8), bc = *reinterpret_cast<const float4*>(bb + g * 8 + 4);
@@ -367,7 +362,7 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                                     val.z = pack_half2(clampf(v[g * 8 + 4] + bc.x, lo1, hi1), clampf(v[g * 8 + 5] + bc.y, lo1, hi1));
                                     val.w = pack_half2(clampf(v[g * 8 + 6] + bc.z, lo1, hi1), clampf(v[g * 8 + 7] + bc.w, lo1, hi1));
                                 }
-                                const int g8 = half * 4 + g;
+                                const int g8 = part * 2 + g;
                                 *reinterpret_cast<uint4*>(hbuf + r * 128 + ((g8 ^ (r & 7)) << 4)) = val;
                             }
                         }
@@ -384,19 +379,19 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                 // ---- depthwise 3x3: H -> Hd ---------------------------------------------------------------
                 const uint8_t* hsrc = hbuf + (p.has_expand ? 0 : hc * p.nb1 * kPlane);
                 const int pairs_w = (p.tw + 1) >> 1;
-                for (int item = wt; item < p.th * pairs_w * 8; item += 32 * kWorkWarps) {
-                    const int g8 = item & 7, pr = item >> 3;
+                for (int item = wt; item < p.th * pairs_w * 16; item += 32 * kWorkWarps) {
+                    const int g4 = item & 15, pr = item >> 4;
                     const int oy = pr / pairs_w, ox = (pr - oy * pairs_w) * 2;
                     const bool second = ox + 1 < p.tw;
-                    if (g8 < groups) {
+                    if (g4 < groups) {
                         // the second window of a last, odd pair reads columns past the frame row: still inside the
                         // buffer (next row or slack), and its result is not stored
-                        if (p.stride == 1) dw_pair<1>(hsrc, hdbuf, p.fw, p.tw, g8, oy, ox, second, wreg, breg, lo2, hi2);
-                        else dw_pair<2>(hsrc, hdbuf, p.fw, p.tw, g8, oy, ox, second, wreg, breg, lo2, hi2);
+                        if (p.stride == 1) dw_pair<1>(hsrc, hdbuf, p.fw, p.tw, g4, oy, ox, second, wreg, breg, lo2, hi2);
+                        else dw_pair<2>(hsrc, hdbuf, p.fw, p.tw, g4, oy, ox, second, wreg, breg, lo2, hi2);
                     } else {  // channel groups the chunk does not have: zero operand columns
-                        const int o = oy * p.tw + ox;
-                        *reinterpret_cast<uint4*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
-                        if (second) *reinterpret_cast<uint4*>(hdbuf + (o + 1) * 128 + ((g8 ^ ((o + 1) & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+                        const int o = oy * p.tw + ox, g8 = g4 >> 1, sub = (g4 & 1) * 8;
+                        *reinterpret_cast<uint2*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4) + sub) = make_uint2(0u, 0u);
+                        if (second) *reinterpret_cast<uint2*>(hdbuf + (o + 1) * 128 + ((g8 ^ ((o + 1) & 7)) << 4) + sub) = make_uint2(0u, 0u);
                     }
                 }
                 fence_proxy_async_smem();  // the projection UMMAs read Hd through the async proxy
@@ -421,7 +416,7 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                     const int o = b * 128 + q * 32 + lane;
                     const bool live = o < p.th * p.tw;   // rows past the image are clipped by the TMA store
                     const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + p.d2_col + b * p.n2_pad;
-                    for (int c0 = half * 16; c0 < p.n2_pad; c0 += 32) {
+                    for (int c0 = part * 16; c0 < p.n2_pad; c0 += 64) {
                         float v[16];
                         __syncwarp();
                         tmem_ld16(taddr + c0, v);
@@ -465,7 +460,7 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                 const bool live = o < p.th * p.tw && gy < p.Ho && gx < p.Wo;
                 const long long gpix = (static_cast<long long>(n) * p.Ho + gy) * p.Wo + gx;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + p.d2_col + b * p.n2_pad;
-                for (int c0 = half * 16; c0 < p.n2_pad; c0 += 32) {
+                for (int c0 = part * 16; c0 < p.n2_pad; c0 += 64) {
                     float v[16];
                     __syncwarp();
                     tmem_ld16(taddr + c0, v);
