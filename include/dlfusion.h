@@ -205,8 +205,13 @@ const char* dlf_net_group_kernel(const dlf_net* net, int group);
  *                               0: launch the kernels one by one.  Does not clear the plan.
  *   DLF_OPT_PDL              1 (default): the tensor-core kernels are launched with programmatic
  *                               dependent launch, so that a kernel's set-up overlaps the tail of
- *                               its predecessor; 0: plain stream order.  Process-wide. */
-enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4, DLF_OPT_PDL = 5 };
+ *                               its predecessor; 0: plain stream order.  Process-wide.
+ *   DLF_OPT_CONV_ROW_MODE    1 (default): a single 3x3 stride-1 convolution whose C_in is a multiple of 64 and
+ *                               whose image is at most 126 pixels wide loads a kernel row's input window once for
+ *                               its three taps where that cuts the bytes a CTA streams by a fifth; 0: never (one
+ *                               window load per tap); 2: wherever it applies.  Process-wide; does not clear the plan. */
+enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4, DLF_OPT_PDL = 5,
+       DLF_OPT_CONV_ROW_MODE = 6 };
 int dlf_net_set_option(dlf_net* net, int option, int value);
 
 /* Size of the scratch array that dlf_conv_chain_run_static keeps inside the library image. */

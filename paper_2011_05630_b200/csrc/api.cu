@@ -18,6 +18,7 @@ namespace dlf {
 
 static thread_local int g_last_cuda_error = 0;
 int g_use_pdl = 1;
+int g_conv_row_mode = 1;
 
 int cuda_fail(cudaError_t e) {
     g_last_cuda_error = static_cast<int>(e);
@@ -1078,6 +1079,11 @@ int dlf_net_set_option(dlf_net* net, int option, int value) {
         case DLF_OPT_SINGLE_AS_CHAIN: net->opt_single_chain = value != 0; break;
         case DLF_OPT_CUDA_GRAPH: net->opt_graph = value != 0; return DLF_OK;
         case DLF_OPT_PDL: g_use_pdl = value != 0; invalidate_graphs(net); return DLF_OK;
+        case DLF_OPT_CONV_ROW_MODE:
+            if (value < 0 || value > 2) return DLF_E_INVALID_ARG;
+            g_conv_row_mode = value;
+            invalidate_graphs(net);
+            return DLF_OK;
         default: return DLF_E_INVALID_ARG;
     }
     net->plan.clear();  // kernel choices depend on the options: the plan must be set again

@@ -596,7 +596,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     Tile tl_row{};
     int bias_row = 0;
     double cost_row = 0.0;
-    if (a.kh == 3 && a.kw == 3 && a.stride == 1 && a.pad == 1 && !a.pool && p.grouped && a.Wo + 2 <= 128 && a.W == a.Wo && a.H == a.Ho) {
+    if (g_conv_row_mode > 0 && a.kh == 3 && a.kw == 3 && a.stride == 1 && a.pad == 1 && !a.pool && p.grouped && a.Wo + 2 <= 128 && a.W == a.Wo && a.H == a.Ho) {
         const int th_row = std::min(a.Ho, 128 / (a.Wo + 2));
         // several whole images per tile where they fit (an image's rows stay together, so the shifted reads of its
         // valid pixels never reach the next image)
@@ -609,7 +609,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     }
     set_tile(pick_tile(a.N, a.Ho, a.Wo, a.pool), 1);
     if (!configure(kMaxSmem, 256, 1)) return DLF_E_UNSUPPORTED;
-    if (row_mode && cost_row < 0.8 * stream_cost()) {
+    if (row_mode && (g_conv_row_mode > 1 || cost_row < 0.8 * stream_cost())) {
         const long long keep_m = static_cast<long long>(p_row.tiles_w) * p_row.tiles_h * p_row.tiles_n;
         p = p_row; tl = tl_row; bias_bytes = bias_row; m_tiles = keep_m;
     }

@@ -65,6 +65,7 @@ int chain_tc_init();
 // Launches a kernel, optionally with programmatic dependent launch (the kernel must then call
 // pdl_wait() before it touches anything its predecessor in the stream produces).
 extern int g_use_pdl;
+extern int g_conv_row_mode;  // conv_tc row mode: 0 never, 1 where it cuts the streamed bytes by a fifth, 2 wherever it applies
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_kernel(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t s, Args... args) {
     cudaLaunchConfig_t cfg = {};

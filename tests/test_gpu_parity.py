@@ -90,6 +90,40 @@ def test_single_layer(case):
         assert sess.kernels() == ["chain_tc"]
 
 
+ROW_MODE = [
+    # 3x3 stride-1 layers through the row mode of the single-layer kernel (forced), then with it switched off
+    (3, 9, 13, _conv(64, 128, 3)),                    # two tiles per image, the second one a single row
+    (5, 7, 7, _conv(128, 64, 3, act="none")),        # two whole images per tile, ragged batch
+    (1, 5, 126, _conv(64, 128, 3, act="relu6")),     # widest image: pitch 128, one row per tile
+    (1, 6, 127, _conv(64, 128, 3)),                   # one pixel wider: no row mode, one window load per tap
+    (2, 28, 28, _conv(192, 320, 3)),                  # three chunks, two channel tiles (the second one narrower)
+]
+
+
+@pytest.mark.parametrize("case", ROW_MODE, ids=lambda c: "%dx%dx%d_%d_%d" % (c[0], c[1], c[2], c[3]["cin"], c[3]["cout"]))
+def test_single_3x3_layer_row_mode_on_and_off(case):
+    n, h, w, layer = case
+    sess, xd, ref = _mk([layer], "rowmode", n, h, w, layer["cin"])
+    try:
+        for mode in (2, 0):
+            B.net_set_option(sess.net, B.OPT_CONV_ROW_MODE, mode)
+            for s in (sms(), 5):
+                G.check_plan(sess, xd, ref, [0], [s], "row mode %d S=%d" % (mode, s))
+            assert sess.kernels() == ["conv_tc"]
+    finally:
+        B.net_set_option(sess.net, B.OPT_CONV_ROW_MODE, 1)
+
+
+def test_row_mode_with_residual():
+    layers = [_conv(64, 128, 1, act="none"), _conv(128, 128, 3, src=0, res_src=0)]
+    sess, xd, ref = _mk(layers, "rowres", 3, 14, 14, 64)
+    try:
+        B.net_set_option(sess.net, B.OPT_CONV_ROW_MODE, 2)
+        G.check_plan(sess, xd, ref, [0, 1], [sms(), sms()], "row mode residual")
+    finally:
+        B.net_set_option(sess.net, B.OPT_CONV_ROW_MODE, 1)
+
+
 def test_single_layer_with_residual_through_both_conv_kernels():
     layers = [_conv(64, 64, 1, act="none"), _conv(64, 64, 3, src=0, res_src=-1)]
     sess, xd, ref = _mk(layers, "res", 2, 17, 18, 64)
