@@ -1,6 +1,10 @@
 """Runs one convolution layer a few times through the C ABI (for profiler captures and quick checks).
 
     python -m paper_2011_05630_b200.layer_cli N H W CIN COUT K [--as-chain] [--reps 3] [--stride 1]
+                                              [--op conv|dwconv|maxpool] [--mbconv HID]
+
+--op dwconv runs a depthwise KxK layer (COUT = CIN), --op maxpool a KxK max-pool; --mbconv HID runs the fused
+inverted-residual block CIN -> HID (1x1) -> depthwise 3x3 (--stride) -> COUT (1x1) as one group.
 """
 from __future__ import annotations
 
@@ -16,20 +20,35 @@ def main():
     ap.add_argument("--as-chain", action="store_true", help="use the fused-chain kernel for the single layer")
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--stride", type=int, default=1)
+    ap.add_argument("--op", default="conv", choices=["conv", "dwconv", "maxpool"])
+    ap.add_argument("--mbconv", type=int, default=0, help="hidden width of a fused inverted-residual block")
     a = ap.parse_args()
     from . import binding as B
     from .runtime import Session
-    layer = dict(op="conv", act="relu", cin=a.cin, cout=a.cout, kh=a.k, kw=a.k, stride=a.stride, pad=a.k // 2, groups=1,
-                 src=-1, res_src=-2, pool=0)
+    def mk(op, cin, cout, k, stride, src, act="relu", res=-2):
+        return dict(op=op, act=act, cin=cin, cout=cout, kh=k, kw=k, stride=stride, pad=k // 2, groups=cin if op == "dwconv" else 1,
+                    src=src, res_src=res, pool=0)
+    if a.mbconv:
+        res = -1 if (a.stride == 1 and a.cin == a.cout) else -2
+        layers = [mk("conv", a.cin, a.mbconv, 1, 1, -1, "relu6"), mk("dwconv", a.mbconv, a.mbconv, 3, a.stride, 0, "relu6"),
+                  mk("conv", a.mbconv, a.cout, 1, 1, 1, "none", res)]
+    else:
+        layers = [mk(a.op, a.cin, a.cin if a.op != "conv" else a.cout, a.k, a.stride, -1, "none" if a.op == "maxpool" else "relu")]
     rng = np.random.default_rng(0)
-    params = [((rng.standard_normal((a.cout, a.k, a.k, a.cin)) * (a.k * a.k * a.cin) ** -0.5).astype(np.float16),
-               (rng.standard_normal(a.cout) * 0.1).astype(np.float32))]
+    params = []
+    for l in layers:
+        if l["op"] == "maxpool":
+            params.append(None)
+            continue
+        cg = l["cin"] // l["groups"]
+        params.append(((rng.standard_normal((l["cout"], l["kh"], l["kw"], cg)) * (l["kh"] * l["kw"] * cg) ** -0.5).astype(np.float16),
+                       (rng.standard_normal(l["cout"]) * 0.1).astype(np.float32)))
     x = rng.uniform(-1, 1, (a.n, a.h, a.w, a.cin)).astype(np.float16)
-    sess = Session([layer], params, a.n, a.h, a.w, a.cin)
+    sess = Session(layers, params, a.n, a.h, a.w, a.cin)
     xd = sess.upload(x)
     B.net_set_option(sess.net, B.OPT_CUDA_GRAPH, 0)
     B.net_set_option(sess.net, B.OPT_SINGLE_AS_CHAIN, 1 if a.as_chain else 0)
-    sess.set_plan([0], [B.device_sm_count()])
+    sess.set_plan([len(layers) - 1], [B.device_sm_count()])
     for _ in range(a.reps):
         sess.run(xd)
     print("ran", sess.kernels(), "x", a.reps)
