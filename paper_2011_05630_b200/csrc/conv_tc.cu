@@ -499,11 +499,21 @@ bool conv_tc_supported(const ConvArgs& a) {
     return true;
 }
 
-int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s) {
-    if (!conv_tc_supported(a)) return DLF_E_UNSUPPORTED;
+int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStream_t s) {
+    if (!conv_tc_supported(a_in)) return DLF_E_UNSUPPORTED;
     {
         int rc = conv_tc_init();
         if (rc) return rc;
+    }
+    // A 1x1 stride-1 convolution has no spatial structure: its N x H x W pixels are one list, cut into tiles of any
+    // length, so that the persistent grid's rounds can be filled evenly (below) whatever the image size.
+    ConvArgs a = a_in;
+    const long long flat_pixels = static_cast<long long>(a_in.N) * a_in.H * a_in.W;
+    // (measured to pay for the output-bound layers with few input channels; with more, the image-shaped tiles were as fast or faster)
+    const bool flat = a.kh == 1 && a.kw == 1 && a.stride == 1 && a.pad == 0 && !a.pool && flat_pixels < (1ll << 31) && (a.Cin <= 128 || a.H * a.W == 1);
+    if (flat) {
+        a.N = 1; a.H = 1; a.Ho = 1;
+        a.W = a.Wo = static_cast<int>(flat_pixels);
     }
     ConvTcParams p{};
     p.N = a.N; p.Ho = a.Ho; p.Wo = a.Wo; p.Cout = a.Cout;
@@ -607,7 +617,31 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
             p_row = p; tl_row = tl; bias_row = bias_bytes; cost_row = stream_cost();
         }
     }
-    set_tile(pick_tile(a.N, a.Ho, a.Wo, a.pool), 1);
+    if (flat) {
+        // tile length: the least (rounds of the grid) x (cost of an item); an item costs what it streams into shared
+        // memory (pixels and weight slab per 64-channel chunk) plus what it writes (and reads as residual), the
+        // latter weighted by the ratio of an SM's fill rate to its share of the HBM rate, plus a fixed hand-off cost;
+        // the channel-tile width follows from the tile count as for every layer
+        int best_r = 0;
+        long long best_score = -1;
+        for (int r = 128; r >= 32; r--) {
+            set_tile(Tile{std::min(r, a.Wo), 1, 1}, 1);
+            if (!configure(kMaxSmem, 256, 1)) continue;
+            const long long rounds = (m_tiles * p.n_tiles_n + sm_count - 1) / sm_count;
+            const long long item = static_cast<long long>(p.kchunks) * (p.rows + p.BN) * 128 +
+                                   static_cast<long long>(p.rows) * p.BN * 2 * (a.res ? 2 : 1) * 27 / 10 + 40960;
+            const long long score = rounds * item;
+            if (best_score < 0 || score < best_score) {
+                best_score = score;
+                best_r = p.rows;
+            }
+            if (a.Wo <= r) break;
+        }
+        if (best_r == 0) return DLF_E_UNSUPPORTED;
+        set_tile(Tile{best_r, 1, 1}, 1);
+    } else {
+        set_tile(pick_tile(a.N, a.Ho, a.Wo, a.pool), 1);
+    }
     if (!configure(kMaxSmem, 256, 1)) return DLF_E_UNSUPPORTED;
     if (row_mode && (g_conv_row_mode > 1 || cost_row < 0.8 * stream_cost())) {
         const long long keep_m = static_cast<long long>(p_row.tiles_w) * p_row.tiles_h * p_row.tiles_n;
