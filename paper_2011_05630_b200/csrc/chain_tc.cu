@@ -530,7 +530,18 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
     int act_planes = 0;
     for (int l = 0; l < L; l++)
         if (l < L - 1 || a.pool) act_planes = std::max(act_planes, planes_of(pad16(a.cout[l])));
-    const std::vector<int> cand_h = tile_candidates(a.H, a.pool != 0), cand_w = tile_candidates(a.W, a.pool != 0);
+    const std::vector<int> cand_h = tile_candidates(a.H, a.pool != 0);
+    std::vector<int> cand_w = tile_candidates(a.W, a.pool != 0);
+    // tile widths whose frame pitch is a multiple of 8 rows: a shifted operand window whose first row is not a
+    // multiple of 8 rows into the tile straddles two swizzle atoms per 8-row group and costs the tensor core about
+    // twice the shared-memory reads (measured: 85-90 cycles per N = 64 UMMA instead of 48); with such a pitch the
+    // taps of the centre column start on atom boundaries
+    for (int pitch8 = 8; pitch8 <= 256; pitch8 += 8) {
+        const int tw8 = pitch8 - 2 * halo;
+        if (tw8 >= 2 && tw8 <= a.W && (!a.pool || tw8 % 2 == 0)) cand_w.push_back(tw8);
+    }
+    std::sort(cand_w.begin(), cand_w.end());
+    cand_w.erase(std::unique(cand_w.begin(), cand_w.end()), cand_w.end());
     for (int th : cand_h)
         for (int tw : cand_w) {
             const int rows = th + 2 * halo, pitch = tw + 2 * halo;
@@ -556,7 +567,11 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
                     double mma = 0.0;
                     for (int ch = 0; ch < g.n_chunks; ch++) {
                         const int n = std::min(g.chunk_n, g.n_pad - ch * g.chunk_n);
-                        mma += static_cast<double>(g.nb) * ksteps * std::max(32.0 + n / 4.0, n / 2.0);
+                        // operand reads from shared memory: 4 KB of pixels (8 KB where the window straddles swizzle
+                        // atoms: every tap of a 3x3 layer but the centre column's at a pitch that is a multiple of 8,
+                        // else all but the centre tap) and n x 32 bytes of weights, at 128 bytes per clock
+                        const double straddle = a.k[l] == 1 ? 0.0 : (pitch % 8 == 0 ? 6.0 / 9.0 : 8.0 / 9.0);
+                        mma += static_cast<double>(g.nb) * ksteps * std::max(32.0 * (1.0 + straddle) + n / 4.0, n / 2.0);
                     }
                     const double epi = static_cast<double>(g.nb) * (g.n_pad / 32.0) * 220.0;
                     const int passes = g.n_chunks * ((g.nb + g.per_pass - 1) / g.per_pass);
