@@ -187,7 +187,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         }
     } else if (warp >= kProdWarp0) {
         // ---- producers: TMA loads into the stage ring -------------------------------------------
-        if (lane == 0) {
+        // The warp stays converged; lane g loads the stage's g-th 64-channel chunk as a box of its own: the copies
+        // of a stage run side by side (one thread's copies run one after the other) and every chunk starts on a
+        // 1024-byte boundary whatever the tile's row count (a chunk that starts inside a swizzle atom costs the
+        // tensor core twice the shared-memory reads).
+        {
             const int role = warp - kProdWarp0;
             const bool is_b = role >= 2;
             const uint32_t parity = role & 1;
@@ -203,36 +207,43 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     const int r = tap / p.kw, s = tap % p.kw;
                     for (int kq = 0; kq < p.kgroups; kq++, it++) {
                         const int st = it % p.stages;
-                        // a ring stage belongs to ONE producer of each kind: a thread that skipped a phase of
+                        // a ring stage belongs to ONE producer warp of each kind: a warp that skipped a phase of
                         // a stage's barrier could not tell "two phases ago" from "now" by parity
                         if ((st & 1u) != parity) continue;
-                        ok = mbar_wait(&empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status,
-                                       0x100 | (blockIdx.x << 12));
+                        ok = mbar_wait_warp(&empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status,
+                                            0x100 | (blockIdx.x << 12));
                         if (!ok) break;
                         DLF_TRACE_ACC(pacc, 0, pmark);
                         uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
-                        mbar_expect_tx(&full_bar[st], my_bytes);
-                        if (is_b) {
-                            if (p.grouped) tma_load_4d(sa + p.kg * p.a_bytes, &tmw, &full_bar[st], 0, c.co0, tap, kq * p.kg);
-                            else tma_load_3d(sa + p.a_bytes, &tmw, &full_bar[st], kq * 64, tap, c.co0);
-                        } else {
-                            const int wi = c.wo0 * p.stride - p.pad + s, hi = c.ho0 * p.stride - p.pad + r;
-                            if (p.grouped) tma_load_5d(sa, &tmx, &full_bar[st], 0, wi, hi, c.n0, kq * p.kg);
-                            else tma_load_4d(sa, &tmx, &full_bar[st], kq * 64, wi, hi, c.n0);
+                        if (lane == 0) mbar_expect_tx(&full_bar[st], my_bytes);
+                        __syncwarp();
+                        if (lane < p.kg) {   // a chunk past C_in / 64 lies outside the tensor map and arrives as zeros
+                            const int kc = kq * p.kg + lane;
+                            if (is_b) {
+                                uint8_t* dst = sa + p.kg * p.a_bytes + lane * kTps * p.BN * 128;
+                                if (p.grouped) tma_load_4d(dst, &tmw, &full_bar[st], 0, c.co0, tap, kc);
+                                else tma_load_3d(dst, &tmw, &full_bar[st], kc * 64, tap, c.co0);
+                            } else {
+                                const int wi = c.wo0 * p.stride - p.pad + s, hi = c.ho0 * p.stride - p.pad + r;
+                                uint8_t* dst = sa + lane * p.a_bytes;
+                                if (p.grouped) tma_load_5d(dst, &tmx, &full_bar[st], 0, wi, hi, c.n0, kc);
+                                else tma_load_4d(dst, &tmx, &full_bar[st], kc * 64, wi, hi, c.n0);
+                            }
                         }
-                        if (it == 0) DLF_TRACE_POINT(p.status, 2);
+                        __syncwarp();
+                        if (it == 0 && lane == 0) DLF_TRACE_POINT(p.status, 2);
                         DLF_TRACE_ACC(pacc, 1, pmark);
                     }
                 }
             }
-            DLF_TRACE_FLUSH_N(p.status, pacc, 17 + 2 * role, 2);
+            if (lane == 0) DLF_TRACE_FLUSH_N(p.status, pacc, 17 + 2 * role, 2);
         }
     } else if (warp == kMmaWarp) {
         // ---- MMA issuer: the whole warp walks the loop (warp-uniform addresses), one elected lane issues ----
         const uint32_t idesc = umma_idesc_f16(p.BN);
         const uint64_t desc0 = umma_desc_sw128(0, 0);
         const uint32_t b_chunk16 = static_cast<uint32_t>(p.BN) * 8u;  // one 64-channel weight slab, in 16-byte units
-        const uint32_t a_chunk16 = static_cast<uint32_t>(p.rows) * 8u; // one 64-channel slab of the tile's pixels (a box of kg slabs is dense)
+        const uint32_t a_chunk16 = static_cast<uint32_t>(p.a_bytes) >> 4;  // one 64-channel slab of the tile's pixels (rows rounded up to 8)
         uint32_t it = 0, j = 0;
         bool ok = true;
         DLF_TRACE_DECL(macc, mmark);  // cycles of CTA 0's issuer: 0 accumulator wait, 1 stage wait, 2 issue
@@ -660,20 +671,20 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
     CUtensorMap tmx, tmw, tmy, tmr;
     const uint64_t taps64 = static_cast<uint64_t>(a.kh) * a.kw;
     if (p.grouped) {
-        // input seen as (64 channels, W, H, N, C_in / 64): one box carries kg chunks of a tap's window
+        // input seen as (64 channels, W, H, N, C_in / 64): one box carries one 64-channel chunk of a tap's window
         const uint64_t dims[5] = {64, static_cast<uint64_t>(a.W), static_cast<uint64_t>(a.H), static_cast<uint64_t>(a.N),
                                   static_cast<uint64_t>(a.Cin / 64)};
         const uint64_t strides[4] = {static_cast<uint64_t>(a.Cin) * 2, static_cast<uint64_t>(a.W) * a.Cin * 2,
                                      static_cast<uint64_t>(a.H) * a.W * a.Cin * 2, 128};
         const uint32_t box[5] = {64, static_cast<uint32_t>(tl.tw * a.stride), static_cast<uint32_t>(tl.th * a.stride),
-                                 static_cast<uint32_t>(tl.tn), static_cast<uint32_t>(p.kg)};
+                                 static_cast<uint32_t>(tl.tn), 1};
         const uint32_t es[5] = {1, static_cast<uint32_t>(a.stride), static_cast<uint32_t>(a.stride), 1, 1};
         int rc = encode_tmap(&tmx, a.x, 5, dims, strides, box, es);
         if (rc) return rc;
         // weights [cout][tap][cin] seen as (64 channels, cout, tap, C_in / 64)
         const uint64_t wdims[4] = {64, static_cast<uint64_t>(a.Cout), taps64, static_cast<uint64_t>(a.Cin / 64)};
         const uint64_t wstrides[3] = {taps64 * a.Cin * 2, static_cast<uint64_t>(a.Cin) * 2, 128};
-        const uint32_t wbox[4] = {64, static_cast<uint32_t>(p.BN), static_cast<uint32_t>(p.tps), static_cast<uint32_t>(p.kg)};
+        const uint32_t wbox[4] = {64, static_cast<uint32_t>(p.BN), static_cast<uint32_t>(p.tps), 1};
         const uint32_t wes[4] = {1, 1, 1, 1};
         rc = encode_tmap(&tmw, a.w, 4, wdims, wstrides, wbox, wes);
         if (rc) return rc;
