@@ -141,11 +141,20 @@ static bool chain_layer_ok(const Layer& l) {
 // only while its weights stay small next to the tile it works on.
 constexpr int64_t kMaxFusedWeightBytes = 160 * 1024;
 
-static bool span_is_chain(const dlf_net* net, int first, int last) {
+// The tuner (max_layer_flops > 0) also keeps a layer with more work than that out of multi-layer chains: the fused
+// kernel runs a tile's layers one after the other and recomputes halos, which pays only for layers that are short
+// (Sec. IV-B of the paper finds the same: fusion helps its 0.43 G-operation layer and hurts its 1.72 G-operation
+// one).  Measured here: 1x1 64->64 + 3x3 64->64 at 56x56, batch 32 takes 37 us fused, 31 us as two kernels.
+// A plan given explicitly may still ask for such a chain.
+static const double kTunerMaxFusedFlopsPerSm = 2.0e7;
+
+static bool span_is_chain(const dlf_net* net, int first, int last, double max_layer_flops = 0.0) {
     if (last - first + 1 > kMaxChain) return false;
     if (last > first)
-        for (int i = first; i <= last; i++)
+        for (int i = first; i <= last; i++) {
             if (net->layers[i].w_elems * 2 > kMaxFusedWeightBytes) return false;
+            if (max_layer_flops > 0.0 && static_cast<double>(net->layers[i].flops) > max_layer_flops) return false;
+        }
     const int n = static_cast<int>(net->layers.size());
     for (int i = first; i <= last; i++) {
         const Layer& l = net->layers[i];
@@ -749,6 +758,7 @@ int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_
     const int n = static_cast<int>(net->layers.size());
     double sum_op = 0.0, sum_mp = 0.0;
     int block = 0, start = 0, ng = 0;
+    const double max_fl = kTunerMaxFusedFlopsPerSm * s_max;
     for (int i = 0; i < n; i++) {
         const Layer& l = net->layers[i];
         if (is_param(l)) {
@@ -758,11 +768,11 @@ int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_
         }
         // a block may grow while its layers are, or can still become, a group one kernel runs; it may
         // close only where they already are one (inside an inverted-residual block it keeps growing)
-        bool forced = (i == n - 1) || !(span_is_chain(net, start, i + 1) || span_is_mbconv(net, start, i + 1, true, kTunerMaxHidden));
-        const bool closable = (i == start) || span_is_chain(net, start, i) || span_is_mbconv(net, start, i, false, kTunerMaxHidden);
+        bool forced = (i == n - 1) || !(span_is_chain(net, start, i + 1, max_fl) || span_is_mbconv(net, start, i + 1, true, kTunerMaxHidden));
+        const bool closable = (i == start) || span_is_chain(net, start, i, max_fl) || span_is_mbconv(net, start, i, false, kTunerMaxHidden);
         if (!forced && params->legalise) {
             Group g;
-            if (i + 1 > start && (span_is_chain(net, start, i + 1) || span_is_mbconv(net, start, i + 1, false, kTunerMaxHidden)))
+            if (i + 1 > start && (span_is_chain(net, start, i + 1, max_fl) || span_is_mbconv(net, start, i + 1, false, kTunerMaxHidden)))
                 forced = !make_group(net, start, i + 1, s_max, &g);
         }
         if (block > 0) {

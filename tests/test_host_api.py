@@ -94,14 +94,17 @@ def _chain_layer_ok(l):
             and 8 <= l["cout"] <= 2048)
 
 
-def span_is_chain(layers, first, last):
+def span_is_chain(layers, first, last, ops=None, max_layer_ops=0.0):
     """The structural rule of fusable spans, written from its description: a chain of dense
     stride-1 size-keeping 1x1/3x3 convolutions, each reading its predecessor, pool / residual on
     the last layer only, no intermediate map used anywhere else; at most 8 layers; in a group of
-    several layers no layer's weights exceed 160 KB (they are re-streamed for every tile)."""
+    several layers no layer's weights exceed 160 KB (they are re-streamed for every tile) and, for
+    the tuner, no layer has more than `max_layer_ops` operations."""
     if last - first + 1 > 8:
         return False
     if last > first and any(2 * l["cout"] * l["kh"] * l["kw"] * l["cin"] > 160 * 1024 for l in layers[first:last + 1]):
+        return False
+    if last > first and max_layer_ops > 0 and any(ops[i] > max_layer_ops for i in range(first, last + 1)):
         return False
     for i in range(first, last + 1):
         l = layers[i]
@@ -189,11 +192,13 @@ def test_autotune_equals_restated_algorithm1(name, layers, batch, crit):
     ch = [l["cout"] for l in layers]
     n = len(layers)
 
+    MAX_FUSED_OPS = 2.0e7 * 148   # the tuner keeps layers with more work per SM than 2e7 operations out of multi-layer chains
+
     def can_extend(start, i):   # layers start..i+1 are, or can still become, one fused group
-        return span_is_chain(layers, start, i + 1) or span_is_mbconv(layers, start, i + 1, True, TUNER_MAX_HIDDEN)
+        return span_is_chain(layers, start, i + 1, ops, MAX_FUSED_OPS) or span_is_mbconv(layers, start, i + 1, True, TUNER_MAX_HIDDEN)
 
     def may_close(start, i):    # layers start..i already are a group one kernel runs
-        return i == start or span_is_chain(layers, start, i) or span_is_mbconv(layers, start, i, False, TUNER_MAX_HIDDEN)
+        return i == start or span_is_chain(layers, start, i, ops, MAX_FUSED_OPS) or span_is_mbconv(layers, start, i, False, TUNER_MAX_HIDDEN)
 
     want = model.algorithm1(kinds, ch, ops, dict(P, op_critical=crit),
                             must_close_after=lambda start, i: i == n - 1 or not can_extend(start, i), may_close=may_close)
