@@ -101,7 +101,7 @@ struct dlf_net {
     std::vector<Layer> layers;
     std::vector<Group> plan;
     uint8_t* ws = nullptr;
-    size_t ws_bytes = 0, ws_need = 0, in_off = 0, in_bytes = 0, status_off = 0;
+    size_t ws_bytes = 0, ws_need = 0, in_off = 0, in_bytes = 0, status_off = 0, splitk_off = 0;
     int dev_sms = 0;
     int opt_no_tc = 0, opt_base_offset = 0, opt_single_chain = 0, opt_graph = 1;
     const void* last_out = nullptr;
@@ -114,6 +114,10 @@ struct dlf_net {
 };
 
 namespace dlf {
+
+// Split-K scratch at the end of a net's workspace: 64 KB of counters and 16 MB of fp32 partial tiles.
+constexpr size_t kSplitKCounterBytes = 65536;
+constexpr size_t kSplitKBytes = kSplitKCounterBytes + (16u << 20);
 
 static bool is_param(const Layer& l) { return l.d.op == DLF_CONV || l.d.op == DLF_DWCONV || l.d.op == DLF_FC; }
 
@@ -280,6 +284,10 @@ static ConvArgs conv_args(const dlf_net* net, int i, const void* in_dev, void* o
     a.Cin = l.d.cin; a.Ho = l.ho_pre; a.Wo = l.wo_pre; a.Cout = l.d.cout;
     a.kh = l.d.kh; a.kw = l.d.kw; a.stride = l.d.stride; a.pad = l.d.pad; a.groups = l.d.groups;
     a.act = l.d.act; a.pool = l.d.pool;
+    if (net->ws) {
+        a.splitk_ws = net->ws + net->splitk_off;
+        a.splitk_bytes = kSplitKBytes;
+    }
     return a;
 }
 
@@ -318,6 +326,10 @@ static ConvArgs fc_as_conv_args(const dlf_net* net, int i, const void* in_dev, v
     a.Cin = l.d.cin; a.Ho = 1; a.Wo = 1; a.Cout = l.d.cout;
     a.kh = 1; a.kw = 1; a.stride = 1; a.pad = 0; a.groups = 1;
     a.act = l.d.act; a.pool = 0;
+    if (net->ws) {
+        a.splitk_ws = net->ws + net->splitk_off;
+        a.splitk_bytes = kSplitKBytes;
+    }
     return a;
 }
 
@@ -644,7 +656,8 @@ int dlf_net_create(const dlf_layer_desc* layers, int n_layers, int N, int H, int
         return rc;
     }
     net->status_off = off;
-    net->ws_need = off + 256;
+    net->splitk_off = off + 256;
+    net->ws_need = net->splitk_off + kSplitKBytes;
     *out = net;
     return DLF_OK;
 }
@@ -687,7 +700,8 @@ int dlf_net_bind_workspace(dlf_net* net, void* workspace_dev, size_t bytes) {
     net->ws = static_cast<uint8_t*>(workspace_dev);
     invalidate_graphs(net);
     net->ws_bytes = bytes;
-    cudaError_t e = cudaMemset(net->ws + net->status_off, 0, 256);
+    // the status block and, behind it, the split-K arrival counters (zero between launches)
+    cudaError_t e = cudaMemset(net->ws + net->status_off, 0, 256 + kSplitKCounterBytes);
     if (e != cudaSuccess) return cuda_fail(e);
     return DLF_OK;
 }

@@ -33,6 +33,7 @@
 #include <cuda_fp16.h>
 
 #include <algorithm>
+#include <cstdio>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -49,6 +50,7 @@ constexpr int kStoreWarp = kProdWarp0 + 4;  // and one warp for the TMA stores o
 constexpr int kThreads = 32 * (kEpiWarps + 6);
 constexpr int kABytes = 128 * 128;  // 128 pixels x 64 fp16
 constexpr int kMaxSmem = 232448 - 1024;  // dynamic part: the 227 KB per-CTA limit minus the static barriers
+constexpr size_t kSplitCounterBytes = 65536;  // head of the split-K workspace: arrival counters, then the partial tiles
 
 struct ConvTcParams {
     int N, Ho, Wo, Cout;
@@ -63,6 +65,9 @@ struct ConvTcParams {
     int n_work;
     int stage_out_off, bias_off;  // byte offsets in dynamic shared memory
     int out_bufs, out_buf_bytes;  // staging buffers (1 or 2) and the size of one
+    int splits, kgs;              // split-K: work items per tile and K-chunk groups per item (1 / kgroups without)
+    float* partial;               // split-K: fp32 partial tiles [tile][split][row][acc_stride]
+    int* counters;                // split-K: arrivals per (tile, epilogue warp); zero between launches
     uint32_t tmem_cols;
     const float* bias;
     const __half* res;
@@ -72,10 +77,18 @@ struct ConvTcParams {
 
 struct TileCoord {
     int n0, ho0, wo0, co0;
+    int tile, ks;  // split-K: the tile's number and which share of K this work item takes
 };
 
+template <bool SPLIT = false>
 __device__ __forceinline__ TileCoord decode_work(const ConvTcParams& p, int t) {
     TileCoord c;
+    c.ks = 0;
+    if (SPLIT) {   // the shares of one tile are neighbours in the work list: they run side by side
+        c.ks = t % p.splits;
+        t /= p.splits;
+    }
+    c.tile = t;
     const int nt = t % p.n_tiles_n;
     int mt = t / p.n_tiles_n;
     c.co0 = nt * p.BN;
@@ -86,7 +99,7 @@ __device__ __forceinline__ TileCoord decode_work(const ConvTcParams& p, int t) {
     return c;
 }
 
-template <int ACT, bool POOL, bool RES, bool ROW>
+template <int ACT, bool POOL, bool RES, bool ROW, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
                const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmr, const ConvTcParams p) {
@@ -140,14 +153,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     if (warp < kProdWarp0 + 2 || warp == kStoreWarp) pdl_wait();
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
-    const int taps = p.kh * p.kw;
     const int k_iters = p.tgroups * p.kgroups;
 
     if (warp == kStoreWarp) {
         // ---- staging buffers out (TMA stores) and residual tiles in (TMA loads) ------------------------
         // One lane per 64-channel plane: a thread's bulk copies run one after the other (about 0.3 us each,
         // measured), the copies of different lanes side by side.
-        if (!POOL) {
+        if (!POOL && !SPLIT) {   // (split-K tiles leave through the partial sums in global memory)
             uint8_t* stage_out = stage0 + p.stage_out_off;
             auto planes_of = [&](const TileCoord& c) { return (min(p.BN, ((p.Cout - c.co0) + 15) & ~15) + 63) >> 6; };
             auto fetch_residual = [&](int t, uint32_t b) {
@@ -199,41 +211,46 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             uint32_t it = 0;
             bool ok = true;
             DLF_TRACE_DECL(pacc, pmark);  // cycles of CTA 0's producers: 0 wait for a free stage, 1 issue
-            for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x) {
-                const TileCoord c = decode_work(p, t);
-                for (int tg = 0; tg < p.tgroups && ok; tg++) {
-                    // row mode: tap group tg = kernel row tg, its window loaded once at the row's first tap
-                    const int tap = tg * kTps;
-                    const int r = tap / p.kw, s = tap % p.kw;
-                    for (int kq = 0; kq < p.kgroups; kq++, it++) {
-                        const int st = it % p.stages;
-                        // a ring stage belongs to ONE producer warp of each kind: a warp that skipped a phase of
-                        // a stage's barrier could not tell "two phases ago" from "now" by parity
-                        if ((st & 1u) != parity) continue;
-                        ok = mbar_wait_warp(&empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status,
-                                            0x100 | (blockIdx.x << 12));
-                        if (!ok) break;
-                        DLF_TRACE_ACC(pacc, 0, pmark);
-                        uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
-                        if (lane == 0) mbar_expect_tx(&full_bar[st], my_bytes);
-                        __syncwarp();
-                        if (lane < p.kg) {   // a chunk past C_in / 64 lies outside the tensor map and arrives as zeros
-                            const int kc = kq * p.kg + lane;
-                            if (is_b) {
-                                uint8_t* dst = sa + p.kg * p.a_bytes + lane * kTps * p.BN * 128;
-                                if (p.grouped) tma_load_4d(dst, &tmw, &full_bar[st], 0, c.co0, tap, kc);
-                                else tma_load_3d(dst, &tmw, &full_bar[st], kc * 64, tap, c.co0);
-                            } else {
-                                const int wi = c.wo0 * p.stride - p.pad + s, hi = c.ho0 * p.stride - p.pad + r;
-                                uint8_t* dst = sa + lane * p.a_bytes;
-                                if (p.grouped) tma_load_5d(dst, &tmx, &full_bar[st], 0, wi, hi, c.n0, kc);
-                                else tma_load_4d(dst, &tmx, &full_bar[st], kc * 64, wi, hi, c.n0);
-                            }
-                        }
-                        __syncwarp();
-                        if (it == 0 && lane == 0) DLF_TRACE_POINT(p.status, 2);
-                        DLF_TRACE_ACC(pacc, 1, pmark);
+            // One ring stage: K-chunk group kq of tap group tg (row mode: tap group tg = kernel row tg, its window
+            // loaded once at the row's first tap).  False once a wait has given up.
+            auto load_stage = [&](const TileCoord& c, int tg, int kq) -> bool {
+                const int st = it % p.stages;
+                // a ring stage belongs to ONE producer warp of each kind: a warp that skipped a phase of
+                // a stage's barrier could not tell "two phases ago" from "now" by parity
+                if ((st & 1u) != parity) return true;
+                if (!mbar_wait_warp(&empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status, 0x100 | (blockIdx.x << 12))) return false;
+                DLF_TRACE_ACC(pacc, 0, pmark);
+                const int tap = tg * kTps;
+                const int r = tap / p.kw, s = tap % p.kw;
+                uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
+                if (lane == 0) mbar_expect_tx(&full_bar[st], my_bytes);
+                __syncwarp();
+                if (lane < p.kg) {   // a chunk past C_in / 64 lies outside the tensor map and arrives as zeros
+                    const int kc = kq * p.kg + lane;
+                    if (is_b) {
+                        uint8_t* dst = sa + p.kg * p.a_bytes + lane * kTps * p.BN * 128;
+                        if (p.grouped) tma_load_4d(dst, &tmw, &full_bar[st], 0, c.co0, tap, kc);
+                        else tma_load_3d(dst, &tmw, &full_bar[st], kc * 64, tap, c.co0);
+                    } else {
+                        const int wi = c.wo0 * p.stride - p.pad + s, hi = c.ho0 * p.stride - p.pad + r;
+                        uint8_t* dst = sa + lane * p.a_bytes;
+                        if (p.grouped) tma_load_5d(dst, &tmx, &full_bar[st], 0, wi, hi, c.n0, kc);
+                        else tma_load_4d(dst, &tmx, &full_bar[st], kc * 64, wi, hi, c.n0);
                     }
+                }
+                __syncwarp();
+                if (it == 0 && lane == 0) DLF_TRACE_POINT(p.status, 2);
+                DLF_TRACE_ACC(pacc, 1, pmark);
+                return true;
+            };
+            for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x) {
+                const TileCoord c = decode_work<SPLIT>(p, t);
+                if (SPLIT) {   // this item's share of the tile's (tap group, K-chunk group) list
+                    const int l0 = c.ks * p.kgs, l1 = min(k_iters, l0 + p.kgs);
+                    for (int li = l0; li < l1 && ok; li++, it++) ok = load_stage(c, li / p.kgroups, li % p.kgroups);
+                } else {
+                    for (int tg = 0; tg < p.tgroups && ok; tg++)
+                        for (int kq = 0; kq < p.kgroups && ok; kq++, it++) ok = load_stage(c, tg, kq);
                 }
             }
             if (lane == 0) DLF_TRACE_FLUSH_N(p.status, pacc, 17 + 2 * role, 2);
@@ -254,8 +271,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             DLF_TRACE_ACC(macc, 0, mmark);
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + acc * p.acc_stride;
-            int kq = 0;
-            for (int ki = 0; ki < k_iters; ki++, it++) {
+            int kq = 0, k_end = k_iters;
+            if (SPLIT) {   // this item's share of the (tap group, K-chunk group) list
+                const int l0 = decode_work<SPLIT>(p, t).ks * p.kgs;
+                k_end = min(k_iters - l0, p.kgs);
+                kq = l0 % p.kgroups;
+            }
+            for (int ki = 0; ki < k_end; ki++, it++) {
                 const int st = it % p.stages;
                 ok = mbar_wait_warp(&full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                 if (!ok) break;
@@ -313,7 +335,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         bool ok = true;
         DLF_TRACE_DECL(eacc, emark);  // cycles of CTA 0's first epilogue thread: 0 staging-buffer wait, 1 accumulator wait, 2 drain
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
-            const TileCoord c = decode_work(p, t);
+            const TileCoord c = decode_work<SPLIT>(p, t);
             const uint32_t acc = j & 1u;
             const int n = c.n0 + tn, ho = c.ho0 + th, wo = c.wo0 + tw;
             const bool valid = m < p.rows && n < p.N && ho < p.Ho && wo < p.Wo;
@@ -321,6 +343,71 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             const long long opix = POOL ? (static_cast<long long>(n) * Hp + (ho >> 1)) * Wp + (wo >> 1) : pix;
             const bool writer = valid && (!POOL || (((ho | wo) & 1) == 0 && (ho >> 1) < Hp && (wo >> 1) < Wp));
             const int ncols = min(p.BN, ((p.Cout - c.co0) + 15) & ~15);
+            if constexpr (SPLIT) {
+                // Split-K: this item's raw fp32 sums go to global memory; of the items of one tile, the warp that
+                // arrives last at the (tile, warp) counter adds the shares up in their fixed order (so the result
+                // does not depend on which was last), applies bias and activation and writes the fp16 output.
+                ok = mbar_wait(&tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
+                if (!ok) break;
+                tc_fence_after_sync();
+                const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.acc_stride;
+                const size_t share = static_cast<size_t>(p.rows) * p.acc_stride;   // floats of one item's partial tile
+                float* tile0 = p.partial + static_cast<size_t>(c.tile) * p.splits * share + static_cast<size_t>(min(m, p.rows - 1)) * p.acc_stride;
+                for (int cc = part * 32; cc < ncols; cc += 32 * kEpiParts) {
+                    uint32_t r[32];
+                    __syncwarp();
+                    tmem_ld32_issue(taddr + cc, r);
+                    tmem_ld32_wait(r);
+                    if (m < p.rows) {
+                        float4* dst = reinterpret_cast<float4*>(tile0 + c.ks * share + cc);
+#pragma unroll
+                        for (int g = 0; g < 8; g++)
+                            __stcg(dst + g, make_float4(__uint_as_float(r[4 * g]), __uint_as_float(r[4 * g + 1]), __uint_as_float(r[4 * g + 2]), __uint_as_float(r[4 * g + 3])));
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+                __threadfence();
+                __syncwarp();
+                int* cnt = p.counters + c.tile * kEpiWarps + warp;
+                int old = 0;
+                if (lane == 0) old = atomicAdd(cnt, 1);
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old == p.splits - 1) {
+                    __threadfence();
+                    if (valid) {
+                        for (int cc = part * 32; cc < ncols; cc += 32 * kEpiParts) {
+                            const int nc = min(32, ncols - cc);
+#pragma unroll
+                            for (int g = 0; g < 4; g++) {
+                                if (g * 8 >= nc) break;
+                                const int co = c.co0 + cc + g * 8;
+                                const float4 b0 = *reinterpret_cast<const float4*>(bias_s + co);
+                                const float4 b1 = *reinterpret_cast<const float4*>(bias_s + co + 4);
+                                float a[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+                                const float4* src = reinterpret_cast<const float4*>(tile0 + cc + g * 8);
+                                for (int sp = 0; sp < p.splits; sp++, src += share / 4) {
+                                    const float4 v0 = __ldcg(src), v1 = __ldcg(src + 1);
+                                    a[0] += v0.x; a[1] += v0.y; a[2] += v0.z; a[3] += v0.w;
+                                    a[4] += v1.x; a[5] += v1.y; a[6] += v1.z; a[7] += v1.w;
+                                }
+                                uint4 o;
+                                uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
+#pragma unroll
+                                for (int e = 0; e < 4; e++) {
+                                    const __half2 hv = __floats2half2_rn(act_t<ACT>(a[2 * e]), act_t<ACT>(a[2 * e + 1]));
+                                    ou[e] = *reinterpret_cast<const uint32_t*>(&hv);
+                                }
+                                if (co < p.Cout) *reinterpret_cast<uint4*>(p.out + pix * p.Cout + co) = o;
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) *cnt = 0;   // ready for the next launch
+                }
+                continue;
+            }
             // The residual of this pixel's next 32 channels, four 16-byte loads issued together without a
             // branch (clamped address; `rok` keeps which are real): fetched one column pass ahead, the first
             // before the accumulator is even complete, so that their latency is never waited for.
@@ -482,8 +569,8 @@ typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap
 
 template <int ACT, bool POOL, bool RES>
 KernelFn pick_row(bool row) {
-    if constexpr (POOL) return conv_tc_kernel<ACT, POOL, RES, false>;   // the row mode has no pooled epilogue
-    else return row ? conv_tc_kernel<ACT, POOL, RES, true> : conv_tc_kernel<ACT, POOL, RES, false>;
+    if constexpr (POOL) return conv_tc_kernel<ACT, POOL, RES, false, false>;   // the row mode has no pooled epilogue
+    else return row ? conv_tc_kernel<ACT, POOL, RES, true, false> : conv_tc_kernel<ACT, POOL, RES, false, false>;
 }
 template <int ACT, bool POOL>
 KernelFn pick_res(bool res, bool row) {
@@ -492,6 +579,16 @@ KernelFn pick_res(bool res, bool row) {
 template <int ACT>
 KernelFn pick_pool(bool pool, bool res, bool row) {
     return pool ? pick_res<ACT, true>(res, row) : pick_res<ACT, false>(res, row);
+}
+// split-K variants: layers without pooling or residual
+template <int ACT>
+KernelFn pick_split_row(bool row) {
+    return row ? conv_tc_kernel<ACT, false, false, true, true> : conv_tc_kernel<ACT, false, false, false, true>;
+}
+KernelFn pick_split(int act, bool row) {
+    if (act == 0) return pick_split_row<0>(row);
+    if (act == 1) return pick_split_row<1>(row);
+    return pick_split_row<2>(row);
 }
 KernelFn pick_kernel(int act, bool pool, bool res, bool row) {
     if (act == 0) return pick_pool<0>(pool, res, row);
@@ -536,6 +633,7 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
     Tile tl{};
     long long m_tiles = 0;
     int bias_bytes = 0;
+    int splits = 1;   // split-K shares per tile that configure() lays the channel tiles out for
     auto set_tile = [&](const Tile& t, int taps_per_stage) {
         tl = t;
         p.TW = tl.tw; p.TH = tl.th; p.TN = tl.tn;
@@ -561,7 +659,7 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
             const int width = std::min(bn, cout16);
             const int nt = (cout16 + width - 1) / width;
             if (nt > 1 && width % 64) continue;
-            const long long waves = (m_tiles * nt + sm_count - 1) / sm_count;
+            const long long waves = (m_tiles * nt * splits + sm_count - 1) / sm_count;
             const long long cost = waves * (width + 96);
             if (best_cost < 0 || cost < best_cost) {
                 best_cost = cost;
@@ -570,7 +668,7 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
             }
         }
         if (best_cost < 0) return false;
-        const int out_planes = a.pool ? 0 : (p.BN + 63) / 64;
+        const int out_planes = (a.pool || splits > 1) ? 0 : (p.BN + 63) / 64;   // (split-K tiles are not staged)
         bias_bytes = (p.n_tiles_n * p.BN * 4 + 1023) / 1024 * 1024;
         p.out_buf_bytes = out_planes * kABytes;
         const int b_bytes = p.tps * p.BN * 128;   // the weight slabs of one 64-channel chunk in a stage
@@ -607,6 +705,28 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
         const long long waves = (m_tiles * p.n_tiles_n + sm_count - 1) / sm_count;
         return static_cast<double>(waves) * p.tgroups * p.kchunks * (p.a_bytes + p.tps * p.BN * 128);
     };
+    // Cost of the current layout with `sp` split-K shares per tile: rounds of the grid x cost of a work item, in bytes of
+    // shared-memory fill.  An item is bound by the slower of its fill and its UMMAs (measured per M = 128, K = 16
+    // instruction: max(N / 2, 32 + N / 4) cycles, against 74 bytes per cycle of fill), plus what it writes (and reads as
+    // residual) weighted by the ratio of an SM's fill rate to its share of the HBM rate, plus a fixed hand-off cost; sharing
+    // a tile costs the fp32 partial tile's round trip and a hand-over on top.  Negative: `sp` shares are not possible.
+    const bool can_split = a.splitk_ws && a.splitk_bytes > kSplitCounterBytes && !a.res && !a.pool;
+    auto split_score = [&](int sp) -> long long {
+        const int loads = p.tgroups * p.kgroups;
+        const int per = (loads + sp - 1) / sp;
+        const long long tiles = m_tiles * p.n_tiles_n;
+        const int acc_stride = (p.BN + 31) / 32 * 32;
+        if (sp > 1 && (!can_split || (sp - 1) * per >= loads || per * p.kg * p.tps < 8 || tiles * kEpiWarps * 4 > static_cast<long long>(kSplitCounterBytes) ||
+                       static_cast<unsigned long long>(tiles) * sp * p.rows * acc_stride * 4 > a.splitk_bytes - kSplitCounterBytes))
+            return -1;
+        const long long rounds = (tiles * sp + sm_count - 1) / sm_count;
+        const long long k_item = std::min<long long>(static_cast<long long>(p.tgroups) * p.kchunks, static_cast<long long>(per) * p.kg);   // 64-channel chunk loads
+        const long long fill = k_item * (p.a_bytes + p.tps * p.BN * 128);
+        const long long mma = k_item * p.tps * 4 * std::max(p.BN / 2, 32 + p.BN / 4) * 74;
+        const long long item = std::max(fill, mma) + static_cast<long long>(p.rows) * p.BN * 2 * (a.res ? 2 : 1) * 27 / 10 +
+                               (sp > 1 ? static_cast<long long>(p.rows) * p.BN * 8 * 27 / 10 + 600000 : 0) + 40960;
+        return rounds * item;
+    };
     // Row mode (3x3, stride 1, pad 1): a tile is TH whole output rows seen with a pitch of Wo + 2, pixel-linear like
     // its input window, so that the three taps of a kernel row read ONE loaded window through descriptors that
     // start 0, 1 and 2 pixels (128-byte rows) into it: the window is streamed 3 times per 64-channel chunk instead of
@@ -632,23 +752,30 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
         // tile length: the least (rounds of the grid) x (cost of an item); an item costs what it streams into shared
         // memory (pixels and weight slab per 64-channel chunk) plus what it writes (and reads as residual), the
         // latter weighted by the ratio of an SM's fill rate to its share of the HBM rate, plus a fixed hand-off cost;
-        // the channel-tile width follows from the tile count as for every layer
-        int best_r = 0;
+        // the channel-tile width follows from the tile count as for every layer.
+        // Split-K (few tiles, long K: fully connected layers at small batch, where one work item per tile would leave
+        // SMs idle and be bound by the UMMA issue rate): a tile's K range is shared out over `splits` work items that
+        // leave fp32 partial tiles in the caller's workspace; chosen together with the tile length.
+        int best_r = 0, best_s = 1;
         long long best_score = -1;
         for (int r = 128; r >= 32; r--) {
-            set_tile(Tile{std::min(r, a.Wo), 1, 1}, 1);
-            if (!configure(kMaxSmem, 256, 1)) continue;
-            const long long rounds = (m_tiles * p.n_tiles_n + sm_count - 1) / sm_count;
-            const long long item = static_cast<long long>(p.kchunks) * (p.rows + p.BN) * 128 +
-                                   static_cast<long long>(p.rows) * p.BN * 2 * (a.res ? 2 : 1) * 27 / 10 + 40960;
-            const long long score = rounds * item;
-            if (best_score < 0 || score < best_score) {
-                best_score = score;
-                best_r = p.rows;
+            for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
+                if (sp > 1 && !can_split) break;
+                splits = sp;
+                set_tile(Tile{std::min(r, a.Wo), 1, 1}, 1);
+                if (!configure(kMaxSmem, 256, 1)) continue;
+                const long long score = split_score(sp);
+                if (score < 0) continue;
+                if (best_score < 0 || score < best_score) {
+                    best_score = score;
+                    best_r = p.rows;
+                    best_s = sp;
+                }
             }
             if (a.Wo <= r) break;
         }
         if (best_r == 0) return DLF_E_UNSUPPORTED;
+        splits = best_s;
         set_tile(Tile{best_r, 1, 1}, 1);
     } else {
         set_tile(pick_tile(a.N, a.Ho, a.Wo, a.pool), 1);
@@ -658,7 +785,36 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
         const long long keep_m = static_cast<long long>(p_row.tiles_w) * p_row.tiles_h * p_row.tiles_n;
         p = p_row; tl = tl_row; bias_bytes = bias_row; m_tiles = keep_m;
     }
-    const long long n_work = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n * p.n_tiles_n;
+    if (!flat && can_split && m_tiles * p.n_tiles_n * 2 <= sm_count) {
+        // few work items (small images at small batch): share each tile's (tap, K-chunk) list out as well
+        const bool row = p.tps == 3;
+        const ConvTcParams keep = p;
+        const int keep_bias = bias_bytes;
+        int best_s = 1;
+        long long best_score = -1;
+        for (int sp : {1, 2, 3, 4, 6, 8, 12, 16}) {
+            splits = sp;
+            if (!configure(kMaxSmem, row ? 128 : 256, row ? 2 : 1)) continue;
+            const long long score = split_score(sp);
+            if (score >= 0 && (best_score < 0 || score < best_score)) {
+                best_score = score;
+                best_s = sp;
+            }
+        }
+        splits = best_s;
+        if (best_s == 1 || !configure(kMaxSmem, row ? 128 : 256, row ? 2 : 1)) {
+            splits = 1;
+            p = keep;
+            bias_bytes = keep_bias;
+        }
+    }
+    p.splits = splits;
+    p.kgs = (p.tgroups * p.kgroups + splits - 1) / splits;
+    if (splits > 1) {
+        p.counters = static_cast<int*>(a.splitk_ws);
+        p.partial = reinterpret_cast<float*>(static_cast<uint8_t*>(a.splitk_ws) + kSplitCounterBytes);
+    }
+    const long long n_work = static_cast<long long>(p.tiles_w) * p.tiles_h * p.tiles_n * p.n_tiles_n * splits;
     if (n_work > 0x7fffffffLL) return DLF_E_UNSUPPORTED;
     p.n_work = static_cast<int>(n_work);
     uint32_t cols = 32;
@@ -724,7 +880,12 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
     const int grid = std::max(1, std::min(sm_count, p.n_work));
     // never two of these CTAs on an SM: each may hold all of tensor memory
     const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024 + (kABytes + 256 - p.a_bytes), 120 * 1024);
-    cudaError_t e = launch_kernel(pick_kernel(a.act, a.pool != 0, a.res != nullptr, p.tps == 3), grid, kThreads, smem, s, tmx, tmw, tmy, tmr, p);
+#ifdef DLF_TRACE
+    fprintf(stderr, "conv_tc: tile %dx%dx%d rows %d BN %d x %d splits %d kgs %d kg %d kgroups %d stages %d out_bufs %d work %d grid %d\n", tl.tn, tl.th, tl.tw,
+            p.rows, p.BN, p.n_tiles_n, p.splits, p.kgs, p.kg, p.kgroups, p.stages, p.out_bufs, p.n_work, grid);
+#endif
+    const KernelFn fn = splits > 1 ? pick_split(a.act, p.tps == 3) : pick_kernel(a.act, a.pool != 0, a.res != nullptr, p.tps == 3);
+    cudaError_t e = launch_kernel(fn, grid, kThreads, smem, s, tmx, tmw, tmy, tmr, p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 
@@ -739,6 +900,11 @@ int conv_tc_init() {
                                                              cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
                         if (e != cudaSuccess) return cuda_fail(e);
                     }
+        for (int act = 0; act < 3; act++)
+            for (int row = 0; row < 2; row++) {
+                cudaError_t e = cudaFuncSetAttribute(pick_split(act, row != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+                if (e != cudaSuccess) return cuda_fail(e);
+            }
         attr_set = true;
     }
     return DLF_OK;

@@ -19,6 +19,10 @@ struct ConvArgs {
     void* y;          // [N][Ho][Wo][Cout], or [N][Ho/2][Wo/2][Cout] with pool == 2
     int N, H, W, Cin, Ho, Wo, Cout;
     int kh, kw, stride, pad, groups, act, pool;
+    // Optional device scratch for split-K (fully connected layers at small batch): 64 KB of arrival counters that
+    // are zero between launches, then room for fp32 partial tiles.  Null: every tile is one work item.
+    void* splitk_ws;
+    size_t splitk_bytes;
 };
 
 // A chain of stride-1, size-keeping dense convolutions executed by one kernel.

@@ -124,6 +124,34 @@ def test_row_mode_with_residual():
         B.net_set_option(sess.net, B.OPT_CONV_ROW_MODE, 1)
 
 
+SPLIT_K = [
+    # few tiles and a long K: the tile's K range is shared out over several work items (fp32 partial tiles, last one adds)
+    (1, 7, 7, _conv(512, 512, 3)),                            # row mode, one pixel tile
+    (1, 14, 14, _conv(1024, 256, 1, act="none")),             # image-shaped tiles, two per image
+    (1, 14, 14, _conv(256, 264, 3, stride=2, act="relu6")),   # strided taps, a narrow second channel tile
+    (2, 7, 7, _conv(2048, 512, 1)),
+    (3, 1, 1, _conv(4096, 520, 1)),                           # 1x1 image: the pixel-list tiling
+]
+
+
+@pytest.mark.parametrize("case", SPLIT_K, ids=lambda c: "%dx%dx%d_%d_%d_k%d" % (c[0], c[1], c[2], c[3]["cin"], c[3]["cout"], c[3]["kh"]))
+def test_single_layer_split_k(case):
+    n, h, w, layer = case
+    sess, xd, ref = _mk([layer], "splitk", n, h, w, layer["cin"])
+    for s in (sms(), sms(), 40, 7, sms()):   # repeated: the arrival counters must be back at zero after every launch
+        G.check_plan(sess, xd, ref, [0], [s], "split-K S=%d" % s)
+    assert sess.kernels() == ["conv_tc"]
+
+
+def test_fc_split_k_at_small_batch():
+    fc = lambda cin, cout, act, src: dict(op="fc", act=act, cin=cin, cout=cout, kh=1, kw=1, stride=1, pad=0, groups=1, src=src, res_src=-2, pool=0)
+    layers = [fc(4 * 4 * 256, 520, "relu", -1), fc(520, 24, "none", 0)]
+    sess, xd, ref = _mk(layers, "fcsplit", 9, 4, 4, 256)   # more than 8 rows: the tensor-core kernel takes the first layer
+    for _ in range(3):
+        G.check_plan(sess, xd, ref, [0, 1], [sms(), sms()], "fc split-K")
+    assert sess.kernels()[0] == "conv_tc"
+
+
 def test_single_layer_with_residual_through_both_conv_kernels():
     layers = [_conv(64, 64, 1, act="none"), _conv(64, 64, 3, src=0, res_src=-1)]
     sess, xd, ref = _mk(layers, "res", 2, 17, 18, 64)
