@@ -115,7 +115,9 @@ int dlf_net_set_weights(dlf_net* net, int layer, const void* w_f16_dev, const fl
 
 /* Workspace: staging for the input of dlf_net_run_host, one slot per layer output (the worst
  * case over plans is the unfused plan, where every layer reaches HBM), scratch for split
- * reductions and a status word.  Contents are undefined between runs. */
+ * reductions (fp32 partial tiles and their arrival counters, which bind_workspace zeroes and
+ * every launch leaves at zero) and a status word.  Contents are undefined between runs; runs of
+ * one net must not overlap in time (they share the slots and the scratch). */
 int dlf_net_workspace_bytes(const dlf_net* net, size_t* bytes);
 int dlf_net_bind_workspace(dlf_net* net, void* workspace_dev, size_t bytes);
 
