@@ -152,17 +152,27 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
         // first element sits on an odd half starts one half into its buffer row.  One unconditional
         // clamped load per word, all in flight together; `okm` keeps which halves lie inside the
         // image and the batch (the others become zero when the words are stored).
-        auto load_patch = [&](int t, uint32_t (&pw)[kPatchRegs], uint32_t& okm) {
+        // first output pixel of a tile; decoded once per tile (three divisions) and handed from the patch fetch to the
+        // build to the drain
+        struct TileOrigin { int wo0, ho0, n0; };
+        auto decode = [&](int t) {
+            TileOrigin o;
             int mt = t;
-            const int wo0 = (mt % p.tiles_w) * p.TW;
+            o.wo0 = (mt % p.tiles_w) * p.TW;
             mt /= p.tiles_w;
-            const int ho0 = (mt % p.tiles_h) * p.TH, n0 = (mt / p.tiles_h) * p.TN;
+            o.ho0 = (mt % p.tiles_h) * p.TH;
+            o.n0 = (mt / p.tiles_h) * p.TN;
+            return o;
+        };
+        auto load_patch = [&](const TileOrigin& to, uint32_t (&pw)[kPatchRegs], uint32_t& okm) {
+            const int wo0 = to.wo0, ho0 = to.ho0, n0 = to.n0;
             const int wi0 = wo0 * p.stride - p.pad, hi0 = ho0 * p.stride - p.pad;
             const int tile_base = ((n0 * p.H + hi0) * p.W + wi0) * cin;
             const int h_lo = max(0, -wi0) * cin, h_hi = (p.W - wi0) * cin;   // halves of a patch row inside the image
             okm = 0u;
 #pragma unroll
             for (int i = 0; i < kPatchRegs; i++) {
+                if (i * 32 * kWorkWarps >= p.patch_words) break;   // (uniform) a small patch needs only the first few passes
                 const int wI = meta[i] & 0xFFF, y = (meta[i] >> 12) & 0x3FF, nl = meta[i] >> 22;
                 const int n = n0 + nl, hi_row = hi0 + y;
                 const bool row_ok = n < p.N && hi_row >= 0 && hi_row < p.H;
@@ -177,18 +187,16 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
         auto store_patch = [&](uint32_t* dst, const uint32_t (&pw)[kPatchRegs], uint32_t okm) {
 #pragma unroll
             for (int i = 0; i < kPatchRegs; i++) {
+                if (i * 32 * kWorkWarps >= p.patch_words) break;
                 const int widx = threadIdx.x + i * 32 * kWorkWarps;
                 const uint32_t m = ((okm >> (2 * i)) & 1u ? 0x0000FFFFu : 0u) | ((okm >> (2 * i)) & 2u ? 0xFFFF0000u : 0u);
                 if (widx < p.patch_words) dst[widx] = pw[i] & m;
             }
         };
         // rows of the A tile from the staged patch, CH 16-byte chunks per kernel row
-        auto build_rows = [&](auto ch_tag, int t, uint8_t* abuf, const uint32_t* pbuf) {
+        auto build_rows = [&](auto ch_tag, const TileOrigin& to, uint8_t* abuf, const uint32_t* pbuf) {
             constexpr int CH = decltype(ch_tag)::value;
-            int mt = t;
-            const int wo0 = (mt % p.tiles_w) * p.TW;
-            mt /= p.tiles_w;
-            const int ho0 = (mt % p.tiles_h) * p.TH, n0 = (mt / p.tiles_h) * p.TN;
+            const int wo0 = to.wo0, ho0 = to.ho0, n0 = to.n0;
             const int tile_base = ((n0 * p.H + ho0 * p.stride - p.pad) * p.W + wo0 * p.stride - p.pad) * cin;
             const int sc = p.stride * cin;
 #pragma unroll 2
@@ -216,8 +224,9 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
         };
         uint32_t pw[kPatchRegs];
         uint32_t pok = 0u;
+        TileOrigin cur = decode(blockIdx.x), next = cur, prev = cur;
         if (static_cast<int>(blockIdx.x) < p.n_work) {
-            load_patch(blockIdx.x, pw, pok);
+            load_patch(cur, pw, pok);
             store_patch(patch, pw, pok);
         }
         // the activation as a clamp: none (-inf, inf), ReLU [0, inf), ReLU6 [0, 6]
@@ -237,16 +246,19 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
             const bool have = t < p.n_work;
             const bool have_next = have && t + static_cast<int>(gridDim.x) < p.n_work;
             DLF_TRACE_ACC(tacc, 0, tmark);
-            if (have_next) load_patch(t + gridDim.x, pw, pok);
+            if (have_next) {
+                next = decode(t + gridDim.x);
+                load_patch(next, pw, pok);
+            }
             DLF_TRACE_ACC(tacc, 1, tmark);
             if (have) {
                 uint8_t* abuf = sbase + (j & 1u) * a_bytes;
                 const uint32_t* pbuf = patch + (j & 1u) * p.patch_words;
                 switch (p.KR >> 3) {
-                    case 1: build_rows(std::integral_constant<int, 1>{}, t, abuf, pbuf); break;
-                    case 2: build_rows(std::integral_constant<int, 2>{}, t, abuf, pbuf); break;
-                    case 3: build_rows(std::integral_constant<int, 3>{}, t, abuf, pbuf); break;
-                    default: build_rows(std::integral_constant<int, 4>{}, t, abuf, pbuf); break;
+                    case 1: build_rows(std::integral_constant<int, 1>{}, cur, abuf, pbuf); break;
+                    case 2: build_rows(std::integral_constant<int, 2>{}, cur, abuf, pbuf); break;
+                    case 3: build_rows(std::integral_constant<int, 3>{}, cur, abuf, pbuf); break;
+                    default: build_rows(std::integral_constant<int, 4>{}, cur, abuf, pbuf); break;
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
@@ -259,10 +271,7 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
                 DLF_TRACE_ACC(tacc, 3, tmark);
                 if (!ok) break;
                 tc_fence_after_sync();
-                int mt = prev_t;
-                const int wo0 = (mt % p.tiles_w) * p.TW;
-                mt /= p.tiles_w;
-                const int ho0 = (mt % p.tiles_h) * p.TH, n0 = (mt / p.tiles_h) * p.TN;
+                const int wo0 = prev.wo0, ho0 = prev.ho0, n0 = prev.n0;
                 const int m = q * 32 + lane;
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + b * 64u;
                 uint8_t* sout = stage_out + b * kPlane;   // its previous store was waited for before the last barrier
@@ -296,6 +305,8 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
             }
             if (!have) break;
             prev_t = t;
+            prev = cur;
+            cur = next;
             DLF_TRACE_ACC(tacc, 5, tmark);
             if (have_next) store_patch(patch + ((j + 1) & 1u) * p.patch_words, pw, pok);
             // the staging buffer the next drain writes was read by the store before the newest one
