@@ -94,7 +94,7 @@ struct EpiCtx {
     int b0, nblk, ncols, ch0; // blocks of this pass, columns and first channel of this chunk
     uint8_t* obuf;
     const float* bl;
-    float act_lo, act_hi;
+    __half2 act_lo, act_hi;   // applied to rounded pairs
 };
 
 // Drains one pass.  MODE 0: next layer's operand tile in shared memory (zero outside the image);
@@ -146,12 +146,10 @@ __device__ __forceinline__ void epi_pass(const ChainParams& p, const ChainLayerP
                     }
                     // channels past cout (padding up to 16) carry zero weights and zero bias: act(0) = 0,
                     // so the next layer's K padding stays zero
-#pragma unroll
-                    for (int e = 0; e < 8; e++) a[e] = fminf(fmaxf(a[e], cx.act_lo), cx.act_hi);
-                    val.x = pack_half2(a[0], a[1]);
-                    val.y = pack_half2(a[2], a[3]);
-                    val.z = pack_half2(a[4], a[5]);
-                    val.w = pack_half2(a[6], a[7]);
+                    val.x = pack_half2_clamp(a[0], a[1], cx.act_lo, cx.act_hi);
+                    val.y = pack_half2_clamp(a[2], a[3], cx.act_lo, cx.act_hi);
+                    val.z = pack_half2_clamp(a[4], a[5], cx.act_lo, cx.act_hi);
+                    val.w = pack_half2_clamp(a[6], a[7], cx.act_lo, cx.act_hi);
                 }
                 if (kGlobal) {
                     if (co < L.cout) *reinterpret_cast<uint4*>(p.out + gpix * L.cout + co) = val;
@@ -359,8 +357,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                 const int mode = (last && !p.pool) ? (p.res != nullptr ? 2 : 1) : ((last && p.res != nullptr) ? 3 : 0);
                 cx.obuf = sbase + p.act_off + (l & 1) * p.act_buf_bytes;
                 cx.bl = bias_s + L.bias_off;
-                cx.act_lo = L.act >= 1 ? 0.0f : -INFINITY;
-                cx.act_hi = L.act == 2 ? 6.0f : INFINITY;
+                cx.act_lo = __float2half2_rn(L.act >= 1 ? 0.0f : -INFINITY);
+                cx.act_hi = __float2half2_rn(L.act == 2 ? 6.0f : INFINITY);
                 for (int c = 0; c < L.n_chunks && ok; c++) {
                     cx.ncols = chunk_cols(L, c);
                     cx.ch0 = c * L.chunk_n;

@@ -396,7 +396,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                                 uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
                                 for (int e = 0; e < 4; e++) {
-                                    const __half2 hv = __floats2half2_rn(act_t<ACT>(a[2 * e]), act_t<ACT>(a[2 * e + 1]));
+                                    const __half2 hv = act_h2<ACT>(__floats2half2_rn(a[2 * e], a[2 * e + 1]));
                                     ou[e] = *reinterpret_cast<const uint32_t*>(&hv);
                                 }
                                 if (co < p.Cout) *reinterpret_cast<uint4*>(p.out + pix * p.Cout + co) = o;
@@ -476,7 +476,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
                     for (int e = 0; e < 4; e++) {
-                        __half2 hv = __floats2half2_rn(act_t<ACT>(a[2 * e]), act_t<ACT>(a[2 * e + 1]));
+                        __half2 hv = act_h2<ACT>(__floats2half2_rn(a[2 * e], a[2 * e + 1]));   // (clamped after the rounding: same bits)
                         if (POOL) {  // rounded first, then the max over the 2x2 window held by this warp
                             hv = __hmax2(hv, __shfl_xor_sync(0xffffffffu, hv, 1));
                             hv = __hmax2(hv, __shfl_xor_sync(0xffffffffu, hv, p.TW));

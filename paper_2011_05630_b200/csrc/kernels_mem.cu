@@ -137,7 +137,7 @@ __global__ void __launch_bounds__(128) dw3x3_kernel(ConvArgs a, long long total,
             for (int t = 0; t < 9; t++) w[t][j] = __half2float(wv[j * 9 + t]);
         }
     }
-    const float lo = a.act >= 1 ? 0.0f : -INFINITY, hi = a.act == 2 ? 6.0f : INFINITY;
+    const __half2 lo = __float2half2_rn(a.act >= 1 ? 0.0f : -INFINITY), hi = __float2half2_rn(a.act == 2 ? 6.0f : INFINITY);   // applied to rounded pairs
     const __half* x = static_cast<const __half*>(a.x);
     const __half* res = static_cast<const __half*>(a.res);
     __half* y = static_cast<__half*>(a.y);
@@ -211,7 +211,7 @@ __global__ void __launch_bounds__(128) dw3x3_kernel(ConvArgs a, long long total,
             uint32_t* ou = reinterpret_cast<uint32_t*>(&outv);
 #pragma unroll
             for (int e = 0; e < 4; e++)
-                ou[e] = pack_half2(fminf(fmaxf(v[2 * e], lo), hi), fminf(fmaxf(v[2 * e + 1], lo), hi));
+                ou[e] = pack_half2_clamp(v[2 * e], v[2 * e + 1], lo, hi);
             *reinterpret_cast<uint4*>(y + off) = outv;
         }
     }

@@ -64,13 +64,12 @@ struct MbParams {
 
 __device__ __forceinline__ void work_bar_sync() { asm volatile("bar.sync 1, %0;" ::"n"(32 * kWorkWarps) : "memory"); }
 
-__device__ __forceinline__ float clampf(float v, float lo, float hi) { return fminf(fmaxf(v, lo), hi); }
 
 // Depthwise 3x3 of one 4-channel group (8 bytes of a pixel's 128-byte row; g4 = 0..15) for two horizontally
 // adjacent output pixels: the input vectors the two windows share are read from shared memory and converted once.
 template <int STRIDE>
 __device__ __forceinline__ void dw_pair(const uint8_t* hsrc, uint8_t* hdbuf, int fw, int tw, int g4, int oy, int ox, bool second,
-                                        const float (&wreg)[9][4], const float (&breg)[4], float lo, float hi) {
+                                        const float (&wreg)[9][4], const float (&breg)[4], __half2 lo, __half2 hi) {
     constexpr int kCols = STRIDE + 3;  // input columns the two windows cover
     const int g8 = g4 >> 1, sub = (g4 & 1) * 8;
     float acc[2][4];
@@ -102,8 +101,8 @@ __device__ __forceinline__ void dw_pair(const uint8_t* hsrc, uint8_t* hdbuf, int
         if (k == 1 && !second) break;
         const int o = oy * tw + ox + k;
         uint2 val;
-        val.x = pack_half2(clampf(acc[k][0] + breg[0], lo, hi), clampf(acc[k][1] + breg[1], lo, hi));
-        val.y = pack_half2(clampf(acc[k][2] + breg[2], lo, hi), clampf(acc[k][3] + breg[3], lo, hi));
+        val.x = pack_half2_clamp(acc[k][0] + breg[0], acc[k][1] + breg[1], lo, hi);
+        val.y = pack_half2_clamp(acc[k][2] + breg[2], acc[k][3] + breg[3], lo, hi);
         *reinterpret_cast<uint2*>(hdbuf + o * 128 + ((g8 ^ (o & 7)) << 4) + sub) = val;
     }
 }
@@ -295,9 +294,9 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
         // ---- work warps: epilogue 1, depthwise, epilogue 2 ---------------------------------------------------
         const int wt = threadIdx.x;  // 0..255
         const int q = warp & 3, part = warp >> 2;   // TMEM lane quarter; which 16-column slice of every 64 columns
-        const float lo1 = p.act1 >= 1 ? 0.0f : -INFINITY, hi1 = p.act1 == 2 ? 6.0f : INFINITY;
-        const float lo2 = p.act2 >= 1 ? 0.0f : -INFINITY, hi2 = p.act2 == 2 ? 6.0f : INFINITY;
-        const float lo3 = p.act3 >= 1 ? 0.0f : -INFINITY, hi3 = p.act3 == 2 ? 6.0f : INFINITY;
+        const __half2 lo1 = __float2half2_rn(p.act1 >= 1 ? 0.0f : -INFINITY), hi1 = __float2half2_rn(p.act1 == 2 ? 6.0f : INFINITY);
+        const __half2 lo2 = __float2half2_rn(p.act2 >= 1 ? 0.0f : -INFINITY), hi2 = __float2half2_rn(p.act2 == 2 ? 6.0f : INFINITY);
+        const __half2 lo3 = __float2half2_rn(p.act3 >= 1 ? 0.0f : -INFINITY), hi3 = __float2half2_rn(p.act3 == 2 ? 6.0f : INFINITY);
         uint8_t* hbuf = sb + (p.has_expand ? p.h_off : p.x_off);
         uint8_t* hdbuf = sb + p.hd_off;
         uint32_t ti = 0, cc = 0;
@@ -357,10 +356,10 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                                 uint4 val = make_uint4(0u, 0u, 0u, 0u);
                                 if (in_img) {
                                     const float4 ba = *reinterpret_cast<const float4*>(bb + g * 8), bc = *reinterpret_cast<const float4*>(bb + g * 8 + 4);
-                                    val.x = pack_half2(clampf(v[g * 8 + 0] + ba.x, lo1, hi1), clampf(v[g * 8 + 1] + ba.y, lo1, hi1));
-                                    val.y = pack_half2(clampf(v[g * 8 + 2] + ba.z, lo1, hi1), clampf(v[g * 8 + 3] + ba.w, lo1, hi1));
-                                    val.z = pack_half2(clampf(v[g * 8 + 4] + bc.x, lo1, hi1), clampf(v[g * 8 + 5] + bc.y, lo1, hi1));
-                                    val.w = pack_half2(clampf(v[g * 8 + 6] + bc.z, lo1, hi1), clampf(v[g * 8 + 7] + bc.w, lo1, hi1));
+                                    val.x = pack_half2_clamp(v[g * 8 + 0] + ba.x, v[g * 8 + 1] + ba.y, lo1, hi1);
+                                    val.y = pack_half2_clamp(v[g * 8 + 2] + ba.z, v[g * 8 + 3] + ba.w, lo1, hi1);
+                                    val.z = pack_half2_clamp(v[g * 8 + 4] + bc.x, v[g * 8 + 5] + bc.y, lo1, hi1);
+                                    val.w = pack_half2_clamp(v[g * 8 + 6] + bc.z, v[g * 8 + 7] + bc.w, lo1, hi1);
                                 }
                                 const int g8 = part * 2 + g;
                                 *reinterpret_cast<uint4*>(hbuf + r * 128 + ((g8 ^ (r & 7)) << 4)) = val;
@@ -441,10 +440,10 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                                 }
                             }
                             uint4 val;
-                            val.x = pack_half2(clampf(a[0], lo3, hi3), clampf(a[1], lo3, hi3));
-                            val.y = pack_half2(clampf(a[2], lo3, hi3), clampf(a[3], lo3, hi3));
-                            val.z = pack_half2(clampf(a[4], lo3, hi3), clampf(a[5], lo3, hi3));
-                            val.w = pack_half2(clampf(a[6], lo3, hi3), clampf(a[7], lo3, hi3));
+                            val.x = pack_half2_clamp(a[0], a[1], lo3, hi3);
+                            val.y = pack_half2_clamp(a[2], a[3], lo3, hi3);
+                            val.z = pack_half2_clamp(a[4], a[5], lo3, hi3);
+                            val.w = pack_half2_clamp(a[6], a[7], lo3, hi3);
                             *sp = val;
                         }
                     }
@@ -483,10 +482,10 @@ __global__ void __launch_bounds__(kThreads, 1) mbconv_tc_kernel(const __grid_con
                             }
                         }
                         uint4 val;
-                        val.x = pack_half2(clampf(a[0], lo3, hi3), clampf(a[1], lo3, hi3));
-                        val.y = pack_half2(clampf(a[2], lo3, hi3), clampf(a[3], lo3, hi3));
-                        val.z = pack_half2(clampf(a[4], lo3, hi3), clampf(a[5], lo3, hi3));
-                        val.w = pack_half2(clampf(a[6], lo3, hi3), clampf(a[7], lo3, hi3));
+                        val.x = pack_half2_clamp(a[0], a[1], lo3, hi3);
+                        val.y = pack_half2_clamp(a[2], a[3], lo3, hi3);
+                        val.z = pack_half2_clamp(a[4], a[5], lo3, hi3);
+                        val.w = pack_half2_clamp(a[6], a[7], lo3, hi3);
                         *reinterpret_cast<uint4*>(p.out + gpix * p.Cout + co) = val;
                     }
                 }

@@ -304,5 +304,19 @@ __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
     __half2 h = __floats2half2_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);
 }
+// Two values rounded to fp16, then clamped to [lo, hi] as a pair.  Rounding is monotone and the bounds used (0, 6, the
+// infinities) are fp16 values, so clamping after the rounding gives the same bits as clamping before it - at one
+// instruction per bound and PAIR instead of one per bound and value.
+__device__ __forceinline__ uint32_t pack_half2_clamp(float a, float b, __half2 lo, __half2 hi) {
+    const __half2 h = __hmin2(__hmax2(__floats2half2_rn(a, b), lo), hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+// The activation of a rounded pair: none, ReLU, ReLU6.
+template <int ACT>
+__device__ __forceinline__ __half2 act_h2(__half2 h) {
+    if (ACT >= 1) h = __hmax2(h, __float2half2_rn(0.0f));
+    if (ACT == 2) h = __hmin2(h, __float2half2_rn(6.0f));
+    return h;
+}
 
 }  // namespace dlf

@@ -230,7 +230,9 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
             store_patch(patch, pw, pok);
         }
         // the activation as a clamp: none (-inf, inf), ReLU [0, inf), ReLU6 [0, 6]
-        const float act_lo = p.act == DLF_ACT_NONE ? -INFINITY : 0.0f, act_hi = p.act == DLF_ACT_RELU6 ? 6.0f : INFINITY;
+        // (applied to the rounded pair: rounding is monotone and 0 and 6 are fp16 values, so clamping after the rounding gives
+        // the same bits as before it, at one instruction per two values)
+        const __half2 act_lo = __float2half2_rn(p.act == DLF_ACT_NONE ? -INFINITY : 0.0f), act_hi = __float2half2_rn(p.act == DLF_ACT_RELU6 ? 6.0f : INFINITY);
         // this warp's 32 output channels per pass of the epilogue keep their bias in registers
         float breg[32];
 #pragma unroll
@@ -288,8 +290,10 @@ __global__ void __launch_bounds__(kThreads, 1) stem_tc_kernel(const __grid_const
                         uint32_t* ou = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
                         for (int e = 0; e < 4; e++)
-                            ou[e] = pack_half2(fminf(fmaxf(v[g * 8 + 2 * e] + breg[g * 8 + 2 * e], act_lo), act_hi),
-                                               fminf(fmaxf(v[g * 8 + 2 * e + 1] + breg[g * 8 + 2 * e + 1], act_lo), act_hi));
+                        {
+                            const __half2 hv = __hmin2(__hmax2(__floats2half2_rn(v[g * 8 + 2 * e] + breg[g * 8 + 2 * e], v[g * 8 + 2 * e + 1] + breg[g * 8 + 2 * e + 1]), act_lo), act_hi);
+                            ou[e] = *reinterpret_cast<const uint32_t*>(&hv);
+                        }
                         const int g8 = (cc >> 3) + g;
                         *reinterpret_cast<uint4*>(sout + m * 128 + (((g8 & 7) ^ (m & 7)) << 4)) = o;
                     }
