@@ -848,6 +848,8 @@ int dlf_net_sync(dlf_net* net, void* stream) {
         if (st != 0) {
             g_last_cuda_error = st;
             cudaMemset(net->ws + net->status_off, 0, sizeof(int));
+            // a launch that gave up may have left split-K arrival counters behind
+            cudaMemset(net->ws + net->splitk_off, 0, kSplitKCounterBytes);
             return DLF_E_TIMEOUT;
         }
     }
