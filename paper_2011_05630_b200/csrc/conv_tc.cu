@@ -140,10 +140,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         tmem_alloc(&tmem_base_s, p.tmem_cols);
         tmem_relinquish();
     }
-    {   // bias of every output channel, zero past C_out (the channel tile is padded to 16)
-        const int n_bias = p.n_tiles_n * p.BN;
-        for (int i = threadIdx.x; i < n_bias; i += kThreads) bias_s[i] = i < p.Cout ? __ldg(p.bias + i) : 0.0f;
-    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -331,6 +327,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         const int Hp = POOL ? p.Ho / 2 : p.Ho, Wp = POOL ? p.Wo / 2 : p.Wo;
         uint8_t* stage_out = stage0 + p.stage_out_off;
         const bool issuer = (threadIdx.x == 0);
+        {   // bias of every output channel, zero past C_out (the channel tile is padded to 16): staged by the epilogue
+            // warps alone, after the CTA-wide barrier, so that the producers' first copies do not wait for these loads
+            const int n_bias = p.n_tiles_n * p.BN;
+            for (int i = threadIdx.x; i < n_bias; i += 32 * kEpiWarps) bias_s[i] = i < p.Cout ? __ldg(p.bias + i) : 0.0f;
+            asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+        }
         uint32_t j = 0;
         bool ok = true;
         DLF_TRACE_DECL(eacc, emark);  // cycles of CTA 0's first epilogue thread: 0 staging-buffer wait, 1 accumulator wait, 2 drain
