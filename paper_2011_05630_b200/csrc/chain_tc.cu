@@ -196,10 +196,6 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         tmem_alloc(&tmem_base_s, 512);
         tmem_relinquish();
     }
-    for (int l = 0; l < p.n_layers; l++) {
-        const ChainLayerP& L = p.L[l];
-        for (int i = threadIdx.x; i < L.n_pad; i += kThreads) bias_s[L.bias_off + i] = i < L.cout ? __ldg(L.bias + i) : 0.0f;
-    }
     tc_fence_before_sync();
     __syncthreads();
     tc_fence_after_sync();
@@ -339,6 +335,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     } else {
         // ---- epilogue warps ------------------------------------------------------------------------------------
         const int et = threadIdx.x;  // 0 .. 32*kEpiWarps-1
+        // biases staged by the epilogue warps alone, behind the CTA-wide barrier: the producers' first copies do not
+        // wait for these loads
+        for (int l = 0; l < p.n_layers; l++) {
+            const ChainLayerP& L = p.L[l];
+            for (int i = et; i < L.n_pad; i += 32 * kEpiWarps) bias_s[L.bias_off + i] = i < L.cout ? __ldg(L.bias + i) : 0.0f;
+        }
+        epi_bar_sync();
         EpiCtx cx;
         cx.row = (warp & 3) * 32 + lane;
         cx.half = warp >> 2;
