@@ -192,12 +192,6 @@ const char* dlf_net_group_kernel(const dlf_net* net, int group);
 /* Options (debugging and ablation); setting one clears the plan, which must be set again.
  *   DLF_OPT_NO_TENSOR_CORE   1: route every dense convolution to the CUDA-core direct kernel
  *                               (multi-layer groups then become illegal).
- *   DLF_OPT_DESC_BASE_OFFSET 0 (default): the fused kernel's shifted shared-memory descriptors
- *                               leave the base-offset field zero (the tensor core applies the
- *                               128-byte swizzle to absolute shared-memory address bits, as the
- *                               TMA unit does when it writes the tile); 1: store the row phase
- *                               of the start address there (gives wrong results on B200; kept
- *                               only to document the measurement).
  *   DLF_OPT_SINGLE_AS_CHAIN  1: a single stride-1 1x1 / 3x3 convolution with <= 256 output
  *                               channels runs through the fused-chain kernel (input tile
  *                               loaded once) instead of the per-tap kernel.
@@ -212,7 +206,7 @@ const char* dlf_net_group_kernel(const dlf_net* net, int group);
  *                               whose image is at most 126 pixels wide loads a kernel row's input window once for
  *                               its three taps where that cuts the bytes a CTA streams by a fifth; 0: never (one
  *                               window load per tap); 2: wherever it applies.  Process-wide; does not clear the plan. */
-enum { DLF_OPT_NO_TENSOR_CORE = 1, DLF_OPT_DESC_BASE_OFFSET = 2, DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4, DLF_OPT_PDL = 5,
+enum { DLF_OPT_NO_TENSOR_CORE = 1, /* 2 is unused */ DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4, DLF_OPT_PDL = 5,
        DLF_OPT_CONV_ROW_MODE = 6 };
 int dlf_net_set_option(dlf_net* net, int option, int value);
 

@@ -14,7 +14,7 @@ OK, E_INVALID_ARG, E_SHAPE, E_PLAN, E_WORKSPACE, E_UNSUPPORTED, E_CUDA, E_TIMEOU
     0, -1, -2, -3, -4, -5, -6, -7, -8)
 OPS = {"conv": 0, "dwconv": 1, "fc": 2, "maxpool": 3, "gavgpool": 4}
 ACTS = {"none": 0, "relu": 1, "relu6": 2}
-OPT_NO_TENSOR_CORE, OPT_DESC_BASE_OFFSET, OPT_SINGLE_AS_CHAIN, OPT_CUDA_GRAPH, OPT_PDL, OPT_CONV_ROW_MODE = 1, 2, 3, 4, 5, 6
+OPT_NO_TENSOR_CORE, OPT_SINGLE_AS_CHAIN, OPT_CUDA_GRAPH, OPT_PDL, OPT_CONV_ROW_MODE = 1, 3, 4, 5, 6
 
 
 class LayerDesc(C.Structure):

@@ -103,7 +103,7 @@ struct dlf_net {
     uint8_t* ws = nullptr;
     size_t ws_bytes = 0, ws_need = 0, in_off = 0, in_bytes = 0, status_off = 0, splitk_off = 0;
     int dev_sms = 0;
-    int opt_no_tc = 0, opt_base_offset = 0, opt_single_chain = 0, opt_graph = 1;
+    int opt_no_tc = 0, opt_single_chain = 0, opt_graph = 1;
     const void* last_out = nullptr;
     // One CUDA graph per (input, output) pointer pair holds the whole plan; a second, instrumented
     // one records an event after every group for per-group timing.
@@ -402,7 +402,7 @@ static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* 
     switch (g.kind) {
         case K_CHAIN_TC: {
             ChainArgs a = chain_args(net, g.first, g.last, in_dev, y);
-            return launch_chain_tc(a, g.tiling, g.sms, net->opt_base_offset, status, s);
+            return launch_chain_tc(a, g.tiling, g.sms, status, s);
         }
         case K_MBCONV: return launch_mbconv_tc(mbconv_args(net, g.first, g.last, in_dev, y), g.mb_tiling, g.sms, status, s);
         case K_CONV_TC:
@@ -715,10 +715,10 @@ int dlf_net_set_plan(dlf_net* net, int n_groups, const int32_t* group_end, const
     std::vector<Group> plan;
     int rc = validate_plan(net, n_groups, group_end, sm_count, &plan);
     if (rc) return rc;
-    net->plan.swap(plan);
-    invalidate_graphs(net);
     rc = kernels_init();
     if (rc) return rc;
+    net->plan.swap(plan);
+    invalidate_graphs(net);
     return DLF_OK;
 }
 
@@ -1008,11 +1008,12 @@ int dlf_net_bruteforce(dlf_net* net, const dlf_search_params* sp, const void* in
     std::vector<Group> saved = net->plan;
     // fill every layer's slot once so that each candidate group finds its inputs in HBM
     int rc = dlf_net_plan_unfused(net);
-    if (rc) { net->plan = saved; return rc; }
+    if (rc) { net->plan = saved; invalidate_graphs(net); return rc; }
     void* final_out = net->ws + net->layers.back().off;
     rc = dlf_net_run(net, in_dev, final_out, s);
     if (rc == DLF_OK) rc = dlf_net_sync(net, s);
     net->plan = saved;
+    invalidate_graphs(net);   // the graph just built holds the no-fusion plan
     if (rc) return rc;
     cudaEvent_t e0, e1;
     if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return cuda_fail(cudaGetLastError());
@@ -1101,7 +1102,6 @@ int dlf_net_set_option(dlf_net* net, int option, int value) {
     if (!net) return DLF_E_INVALID_ARG;
     switch (option) {
         case DLF_OPT_NO_TENSOR_CORE: net->opt_no_tc = value != 0; break;
-        case DLF_OPT_DESC_BASE_OFFSET: net->opt_base_offset = value != 0; break;
         case DLF_OPT_SINGLE_AS_CHAIN: net->opt_single_chain = value != 0; break;
         case DLF_OPT_CUDA_GRAPH: net->opt_graph = value != 0; return DLF_OK;
         case DLF_OPT_PDL: g_use_pdl = value != 0; invalidate_graphs(net); return DLF_OK;

@@ -74,7 +74,7 @@ struct ChainParams {
     int act_off, act_buf_bytes;
     int ring_off, stages, stage_bytes;
     int bias_off, bias_floats;
-    int pool, base_offset_mode;
+    int pool;
     int cout_last;
     const __half* res;
     __half* out;
@@ -251,7 +251,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         }
     } else if (warp == kMmaWarp) {
         // ---- UMMA issuer: the whole warp walks the loops (warp-uniform addresses), one elected lane issues ----
-        const uint64_t desc0 = umma_desc_sw128(0, 0);
+        const uint64_t desc0 = umma_desc_sw128(0);
         uint32_t wit = 0, tile_i = 0, pass_i = 0, act_i = 0;
         bool ok = true;
         DLF_TRACE_DECL(tacc, tmark);  // cycles of CTA 0's issuer: 0 input wait, 1 layer hand-off wait, 2 accumulator wait, 3 weight wait, 4 issue
@@ -305,7 +305,6 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                                             const uint64_t bd = wd0 + static_cast<uint32_t>(g * L.tg + tt) * w_tap16;
                                             const uint32_t arow0 = aplane + shift * 128;
                                             uint64_t ad = desc0 + (arow0 >> 4);
-                                            if (p.base_offset_mode) ad |= static_cast<uint64_t>((arow0 >> 7) & 7u) << 49;  // 128 rows keep the phase
                                             const uint32_t acc0 = (tap | kc) != 0;
                                             uint32_t d_tmem = d_tmem0;
                                             for (int b = 0; b < nblk; b++, d_tmem += L.slot, ad += (128 * 128) >> 4) {
@@ -599,8 +598,7 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
     return best;
 }
 
-int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int base_offset_mode, int* status_dev,
-                    cudaStream_t s) {
+int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int* status_dev, cudaStream_t s) {
     if (!t.ok) return DLF_E_PLAN;
     {
         int rc = chain_tc_init();
@@ -657,7 +655,6 @@ int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int 
     }
     p.bias_floats = boff;
     p.pool = a.pool;
-    p.base_offset_mode = base_offset_mode;
     p.cout_last = a.cout[a.n_layers - 1];
     p.res = static_cast<const __half*>(a.res);
     p.out = static_cast<__half*>(a.y);
@@ -686,11 +683,13 @@ int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int 
 }
 
 int chain_tc_init() {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices] = {};
+    const int dev = current_device_slot();
+    if (dev < 0) return DLF_E_UNSUPPORTED;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(chain_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return cuda_fail(e);
-        attr_set = true;
+        attr_set[dev] = true;
     }
     return DLF_OK;
 }

@@ -254,7 +254,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     } else if (warp == kMmaWarp) {
         // ---- MMA issuer: the whole warp walks the loop (warp-uniform addresses), one elected lane issues ----
         const uint32_t idesc = umma_idesc_f16(p.BN);
-        const uint64_t desc0 = umma_desc_sw128(0, 0);
+        const uint64_t desc0 = umma_desc_sw128(0);
         const uint32_t b_chunk16 = static_cast<uint32_t>(p.BN) * 8u;  // one 64-channel weight slab, in 16-byte units
         const uint32_t a_chunk16 = static_cast<uint32_t>(p.a_bytes) >> 4;  // one 64-channel slab of the tile's pixels (rows rounded up to 8)
         uint32_t it = 0, j = 0;
@@ -602,7 +602,7 @@ KernelFn pick_kernel(int act, bool pool, bool res, bool row) {
 
 bool conv_tc_supported(const ConvArgs& a) {
     if (a.groups != 1) return false;
-    if (a.Cin % 8 || a.Cout % 8 || a.Cout > 4096) return false;
+    if (a.Cin < 8 || a.Cout < 8 || a.Cin % 8 || a.Cout % 8 || a.Cout > 4096) return false;
     if (a.stride < 1 || a.stride > 2) return false;
     if (a.kh * a.kw > 49) return false;
     if (a.N < 1 || a.Ho < 1 || a.Wo < 1) return false;
@@ -892,8 +892,10 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
 }
 
 int conv_tc_init() {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices] = {};
+    const int dev = current_device_slot();
+    if (dev < 0) return DLF_E_UNSUPPORTED;
+    if (!attr_set[dev]) {
         for (int act = 0; act < 3; act++)
             for (int pool = 0; pool < 2; pool++)
                 for (int res = 0; res < 2; res++)
@@ -907,7 +909,7 @@ int conv_tc_init() {
                 cudaError_t e = cudaFuncSetAttribute(pick_split(act, row != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
-        attr_set = true;
+        attr_set[dev] = true;
     }
     return DLF_OK;
 }

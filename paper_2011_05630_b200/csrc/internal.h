@@ -61,7 +61,16 @@ struct ChainTiling {
 int cuda_fail(cudaError_t e);  // records the error for dlf_last_cuda_error, returns DLF_E_CUDA
 int cuda_fail_drv(int e);
 
-// Sets the kernels' shared-memory attributes once (outside any stream capture).
+// A kernel's shared-memory attribute belongs to a device, not to the process: the *_init functions keep one
+// "done" flag per device, indexed by the current device.  -1: no current device or beyond the table.
+constexpr int kMaxDevices = 64;
+inline int current_device_slot() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
+// Sets the kernels' shared-memory attributes once per device (outside any stream capture).
 int kernels_init();
 int conv_tc_init();
 int chain_tc_init();
@@ -128,8 +137,7 @@ int launch_mbconv_tc(const MbconvArgs& a, const MbconvTiling& t, int sm_count, i
 
 // chain_tc.cu
 ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms);
-int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int base_offset_mode, int* status_dev,
-                    cudaStream_t s);
+int launch_chain_tc(const ChainArgs& a, const ChainTiling& t, int sm_count, int* status_dev, cudaStream_t s);
 
 // tensor map encoding through the driver entry point (no link-time dependency on libcuda)
 int encode_tmap(void* out_map /*CUtensorMap*/, const void* base, int rank, const uint64_t* dims,

@@ -572,11 +572,13 @@ MbconvTiling mbconv_tiling(const MbconvArgs& a, int sm_count) {
 }
 
 int mbconv_tc_init() {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices] = {};
+    const int dev = current_device_slot();
+    if (dev < 0) return DLF_E_UNSUPPORTED;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(mbconv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
         if (e != cudaSuccess) return cuda_fail(e);
-        attr_set = true;
+        attr_set[dev] = true;
     }
     return DLF_OK;
 }

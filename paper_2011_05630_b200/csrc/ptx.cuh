@@ -176,14 +176,13 @@ __device__ __forceinline__ void tc_fence_after_sync() {
 // eight rows per 1024-byte swizzle atom, atoms of consecutive row groups 1024 bytes apart.
 // The swizzle is a function of the absolute shared-memory address (bits 7..9 select the XOR of
 // bits 4..6), so a start address on any 128-byte row of a 1024-byte-aligned buffer is valid with
-// base_offset = 0; measured on B200: a non-zero base offset there breaks the operand.
-__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr, uint32_t base_offset) {
+// base-offset field left at zero.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t saddr) {
     uint64_t d = 0;
     d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);        // start address, 16-byte units
     d |= static_cast<uint64_t>(1) << 16;                        // leading byte offset (unused here)
     d |= static_cast<uint64_t>(1024 >> 4) << 32;                // stride byte offset between row groups
     d |= static_cast<uint64_t>(1) << 46;                        // descriptor version of this architecture
-    d |= static_cast<uint64_t>(base_offset & 7u) << 49;
     d |= static_cast<uint64_t>(2) << 61;                        // 128-byte swizzle
     return d;
 }

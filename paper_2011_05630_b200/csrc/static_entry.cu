@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <cstring>
+#include <mutex>
 
 #include "internal.h"
 
@@ -14,8 +15,8 @@ namespace {
 constexpr size_t kHalfBytes = DLF_STATIC_SCRATCH_BYTES / 2;
 static __device__ __align__(256) unsigned char g_static_scratch[DLF_STATIC_SCRATCH_BYTES + 256];
 
-constexpr int kMaxDevices = 64;
-unsigned char* g_scratch_addr[kMaxDevices];  // device address of the array, per device, once resolved
+unsigned char* g_scratch_addr[dlf::kMaxDevices];  // device address of the array, per device, once resolved
+std::mutex g_scratch_mutex;                  // guards the table above
 
 // In host code `g_static_scratch` is only a handle for the symbol, not a device address: the
 // address a kernel can use has to be asked for, with the device in question current.
@@ -23,7 +24,8 @@ int scratch_address(unsigned char** out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return dlf::cuda_fail(e);
-    if (dev < 0 || dev >= kMaxDevices) return DLF_E_UNSUPPORTED;
+    if (dev < 0 || dev >= dlf::kMaxDevices) return DLF_E_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
     if (!g_scratch_addr[dev]) {
         void* p = nullptr;
         e = cudaGetSymbolAddress(&p, g_static_scratch);
@@ -48,6 +50,8 @@ extern "C" int dlf_conv_chain_run_static(const dlf_layer_desc* layers, int n_lay
     for (int i = 0; i < n_layers; i++) {
         const dlf_layer_desc& d = layers[i];
         if (d.op != DLF_CONV || d.groups != 1 || d.res_src != -2 || d.pool != 0) return DLF_E_UNSUPPORTED;
+        if (d.act < DLF_ACT_NONE || d.act > DLF_ACT_RELU6) return DLF_E_INVALID_ARG;
+        if (d.cin < 8 || d.cout < 8) return DLF_E_SHAPE;
         if (d.src != i - 1 || (i > 0 && d.cin != layers[i - 1].cout)) return DLF_E_SHAPE;
         if (d.kh < 1 || d.kw < 1 || d.stride < 1 || d.pad < 0 || h + 2 * d.pad < d.kh || w + 2 * d.pad < d.kw) return DLF_E_SHAPE;
         if (!w_f16_dev[i] || !bias_dev[i]) return DLF_E_INVALID_ARG;

@@ -406,12 +406,14 @@ bool stem_tc_supported(const ConvArgs& a) {
 }
 
 int stem_tc_init() {
-    static bool attr_set = false;
-    if (!attr_set) {
+    static bool attr_set[kMaxDevices] = {};
+    const int dev = current_device_slot();
+    if (dev < 0) return DLF_E_UNSUPPORTED;
+    if (!attr_set[dev]) {
         cudaError_t e = cudaFuncSetAttribute(stem_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(stem_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem);
         if (e != cudaSuccess) return cuda_fail(e);
-        attr_set = true;
+        attr_set[dev] = true;
     }
     return DLF_OK;
 }

@@ -87,6 +87,23 @@ def test_bad_arguments_and_call_order():
     B.net_destroy(net)
 
 
+@pytest.mark.parametrize("layer,status", [
+    (dict(cout=0), B.E_SHAPE), (dict(cin=0), B.E_SHAPE), (dict(cout=-8), B.E_SHAPE), (dict(act=7), B.E_INVALID_ARG),
+    (dict(act=-1), B.E_INVALID_ARG), (dict(cout=12), B.E_UNSUPPORTED), (dict(pool=2), B.E_UNSUPPORTED),
+    (dict(groups=2), B.E_UNSUPPORTED), (dict(src=0), B.E_SHAPE)])
+def test_allocation_free_entry_rejects_bad_layers_before_any_launch(layer, status):
+    # every refusal below is decided on the host from the descriptors alone: no device call is made (the pointers
+    # are dummies), so the cases run without a GPU
+    import ctypes as C
+    d = _conv(8, 8)
+    d["act"] = B.ACTS[d["act"]]
+    d.update(layer)
+    arr = (B.LayerDesc * 1)(B.LayerDesc(B.OPS["conv"], d["act"], d["cin"], d["cout"], d["kh"], d["kw"], d["stride"], d["pad"],
+                                        d["groups"], d["src"], d["res_src"], d["pool"]))
+    ptrs = (C.c_void_p * 1)(256)
+    assert B.lib().dlf_conv_chain_run_static(arr, 1, 1, 6, 6, 256, ptrs, ptrs, 256, 1, None) == status
+
+
 # ---- the auto-tuner against the restated Algorithm 1 ----------------------------------------------------
 def _chain_layer_ok(l):
     return (l["op"] == "conv" and l["groups"] == 1 and l["stride"] == 1 and l["kh"] == l["kw"] and l["kh"] in (1, 3)

@@ -196,3 +196,54 @@ def test_exhaustive_search_on_a_hand_worked_table():
     assert best == (7.5, [1, 2], [2, 2])
     best = model.best_plan_exhaustive(3, [1, 2], lambda a, e, m: table.get((a, e, m)), max_len=1)
     assert best == (9.0, [0, 1, 2], [2, 2, 2])
+
+
+# ---- hand-worked pins of the readings added to Eq. 5 and Algorithm 1 -----------------------------------
+# alpha = beta = kappa = 1, kappa0 = 0 makes the per-layer count log2(C) + log2(ops): integers for powers of two.
+UNIT = dict(alpha=1.0, beta=1.0, kappa=1.0, kappa0=0.0, s_max=32, op_critical=4.0)
+
+
+def test_eq5_score_against_a_literal_number():
+    # 0.316 * log2(64) + 0.659 * log2(2^30) = 1.896 + 19.77
+    assert model.eq5_score(64, 2 ** 30, 0.316, 0.659) == pytest.approx(21.666, abs=1e-9)
+    assert model.eq5_score(2, 4, 3.0, 0.5) == pytest.approx(4.0)   # 3 * 1 + 0.5 * 2
+
+
+def test_layer_mp_rounding_and_clamps_by_hand():
+    assert model.layer_mp(4, 8, UNIT) == 5                          # 2 + 3
+    half = dict(UNIT, kappa=0.5)
+    assert model.layer_mp(4, 8, half) == 3                          # 2.5 rounds away from zero
+    assert model.layer_mp(4, 2, half) == 2                          # 1.5 -> 2
+    assert model.layer_mp(2, 4, dict(UNIT, kappa=0.5, kappa0=-1.0)) == 1    # 0.5 -> 1
+    assert model.layer_mp(1, 1, UNIT) == 1                          # score 0: lower clamp
+    assert model.layer_mp(4, 8, dict(UNIT, kappa0=-9.0)) == 1       # negative: lower clamp
+    assert model.layer_mp(2 ** 20, 2 ** 20, UNIT) == 32             # 40: upper clamp
+    assert model.layer_mp(2 ** 20, 2 ** 20, dict(UNIT, s_max=148)) == 40
+
+
+def test_algorithm1_deferred_close_by_hand():
+    # per-layer counts 8, 4, 4, 6, 4; critical operation count 4 per core.
+    kinds, ch, ops = [True] * 5, [4] * 5, [2 ** 6, 2 ** 2, 2 ** 2, 2 ** 4, 2 ** 2]
+    # Plain pass: layer 0 alone has 64 / 8 = 8 >= 4 and closes; then 4/4, 8/4, 24/(14/3) = 5.1 closes at 3 with
+    # floor(log2(4.67)) -> 4 cores; the tail closes at 4.
+    assert model.algorithm1(kinds, ch, ops, UNIT) == ([0, 3, 4], [8, 4, 4])
+    # The first block may not close before it holds layers 0..2 (a fusable pattern still growing): it closes at
+    # layer 2 with average (8 + 4 + 4) / 3 = 5.33 -> 4 cores; then 16 / 6 < 4 keeps layer 3 open and
+    # (16 + 4) / ((6 + 4) / 2) = 4 closes at layer 4 with average 5 -> 4 cores.
+    part, mps = model.algorithm1(kinds, ch, ops, UNIT, may_close=lambda start, i: not (start == 0 and i < 2))
+    assert (part, mps) == ([2, 4], [4, 4])
+    # a forced end overrides the deferral
+    part, mps = model.algorithm1(kinds, ch, ops, UNIT, must_close_after=lambda start, i: i == 1,
+                                 may_close=lambda start, i: not (start == 0 and i < 2))
+    assert part[0] == 1 and mps[0] == 4                              # average (8 + 4) / 2 = 6 -> 4
+
+
+def test_algorithm1_top_step_on_a_chip_that_is_not_a_power_of_two():
+    # alpha = 1, beta = 0: the per-layer count is log2(C), clamped to 148 cores
+    p = dict(alpha=1.0, beta=0.0, kappa=1.0, kappa0=0.0, s_max=148, op_critical=1e300)
+    full, almost = 2.0 ** 200, 2.0 ** 147
+    assert model.layer_mp(full, 1, p) == 148 and model.layer_mp(almost, 1, p) == 147
+    part, mps = model.algorithm1([True] * 10, [full] * 10, [1] * 10, p)
+    assert (part, mps) == ([9], [148])                               # average 148: the whole chip
+    part, mps = model.algorithm1([True] * 10, [full] * 9 + [almost], [1] * 10, p)
+    assert (part, mps) == ([9], [128])                               # average 147.9: 2^floor(log2) = 128
