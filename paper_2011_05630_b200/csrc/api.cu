@@ -374,10 +374,9 @@ static bool make_group(const dlf_net* net, int first, int last, int sms, Group* 
     g->tiling = ChainTiling{};
     g->mb_tiling = MbconvTiling{};
     if (first == last) {
-        // A single stride-1 3x3 layer with few channels re-reads its input nine times through the
-        // per-tap kernel; the fused-chain kernel loads the tile once (measured faster up to 64 channels).
-        const dlf_layer_desc& d = net->layers[first].d;
-        const bool prefer_chain = net->opt_single_chain || (d.op == DLF_CONV && d.kh == 3 && d.cin <= 64 && d.cout <= 64);
+        // A single layer runs through the single-layer kernels unless the option asks for the fused-group kernel
+        // (a narrow 3x3 layer: 20.5 us in the single-layer kernel's row mode against 26 us here at 56x56x64, batch 32).
+        const bool prefer_chain = net->opt_single_chain != 0;
         if (!(prefer_chain && !net->opt_no_tc && span_is_chain(net, first, last))) return single_kind(net, first, &g->kind);
     }
     if (net->opt_no_tc) return false;

@@ -45,16 +45,17 @@ struct ChainTiling {
     int th, tw;          // output tile of the last layer (before pooling)
     int halo;            // sum of the layers' paddings
     int pitch, rows;     // frame of the input tile: (th + 2 halo) x (tw + 2 halo), pitch = width
-    int rows_alloc;      // rows one 64-channel plane holds (frame + reach of the last 128-row block)
     int tiles_h, tiles_w, n_tiles;
-    int in_bufs;         // 1 or 2 input frames resident (2 = next tile prefetched during compute)
-    int act_bufs;        // intermediate / staging buffers
-    int act_planes;
+    int in_ring;         // 1: the first layer is 1x1 and its input planes stream through the slots one by one
+    int in_group;        // input planes loaded side by side (one producer round)
+    int in_slots;        // input plane slots in shared memory
+    int out_mode;        // last layer: 0 direct 16-byte stores, 1 staging tile + TMA stores, 2 pooled out of a staging tile
+    int stg_bufs;        // staging buffers (0 for direct stores)
     int stages;          // weight ring depth
     int stage_bytes;
     size_t smem_bytes;
     double redundancy;   // computed / useful multiply-accumulates
-    double cost;         // the tiler's time estimate (arbitrary unit)
+    double cost;         // the tiler's time estimate (SM clocks)
     bool ok;
 };
 

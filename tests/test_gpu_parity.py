@@ -42,7 +42,7 @@ def test_two_layer_group_unfused_and_fused(s):
     s = s or sms()
     sess, xd, ref = _mk(nw.two_layer_group(), "cfg1", 1, 32, 32, 16)
     G.check_plan(sess, xd, ref, [0, 1], [s, s], "cfg1 unfused")
-    assert sess.kernels() == ["chain_tc", "chain_tc"]   # narrow 3x3 layers: tile loaded once
+    assert sess.kernels() == ["conv_tc", "conv_tc"]     # single layers run through the single-layer kernel
     G.check_plan(sess, xd, ref, [1], [s], "cfg1 fused")
     assert sess.kernels() == ["chain_tc"]
     # plan invariance on the device itself: fused and unfused agree to rounding flips
@@ -171,9 +171,7 @@ def test_fc_and_avgpool():
 
 def test_tiny_network_with_every_layer_type():
     layers = _tiny_resnet_like()
-    for l in layers:   # channel counts the vector kernels accept
-        pass
-    layers = [dict(l) for l in layers]
+    layers = [dict(l) for l in layers]   # widened below to channel counts the vector kernels accept
     scale = {3: 3, 4: 8, 8: 16, 16: 32, 5: 8}
     for l in layers:
         l["cin"], l["cout"] = scale[l["cin"]], scale[l["cout"]]
@@ -225,7 +223,11 @@ def test_chain_with_pool_and_residual_and_channel_change():
     sess, xd, ref = _mk(layers, "chain2", 2, 18, 22, 32)
     G.check_plan(sess, xd, ref, [0, 1, 2, 3], [sms()] * 4, "unfused")
     G.check_plan(sess, xd, ref, [2, 3], [sms(), 7], "bottleneck-like + pooled tail")
+    assert sess.kernels() == ["chain_tc", "conv_tc"]
+    B.net_set_option(sess.net, B.OPT_SINGLE_AS_CHAIN, 1)   # the pooled single layer through the fused-group kernel
+    G.check_plan(sess, xd, ref, [2, 3], [sms(), 7], "bottleneck-like + pooled tail, single layer as a group")
     assert sess.kernels() == ["chain_tc", "chain_tc"]
+    B.net_set_option(sess.net, B.OPT_SINGLE_AS_CHAIN, 0)
     # a fused group that ends in a pooled layer, odd image size (the last row / column is dropped)
     layers = [_conv(32, 64, 3), _conv(64, 48, 3, src=0, pool=2), _conv(48, 48, 1, src=1)]
     sess, xd, ref = _mk(layers, "chain3", 2, 19, 21, 32)
