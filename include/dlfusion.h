@@ -133,6 +133,13 @@ int dlf_net_get_plan(const dlf_net* net, int* n_groups, int32_t* group_end, int3
 /* 1 if layers first..last can run as one fused kernel on `sm_count` SMs, 0 if not. */
 int dlf_net_group_is_legal(const dlf_net* net, int first, int last, int sm_count);
 
+/* The rule that bounds Algorithm 1's blocks here (the paper's vendor SDK fuses "almost arbitrary" layers, Sec. III-B; this
+ * library has three fused kernels): 1 if the tuner may propose layers first..last as one group on s_max SMs - the span is
+ * an inverted-residual block up to the measured hidden width, or a dense chain whose fused kernel is estimated (by its own
+ * tiler) to beat one kernel per layer, or, with DLF_OPT_GROUP_KERNEL = 2, any run of dense convolutions.  With prefix != 0
+ * the layers may also be the beginning of an inverted-residual block that can still grow.  0 if not.  Host only. */
+int dlf_net_tuner_may_fuse(const dlf_net* net, int first, int last, int prefix, int s_max);
+
 /* Algorithm 1 with Eq. 5 (host only, O(n)).  Writes the plan into the arrays (n_layers entries
  * each) and does NOT install it; pass it to dlf_net_set_plan. */
 int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_groups,
@@ -185,8 +192,8 @@ int dlf_net_boundary_tensor(const dlf_net* net, int layer, const void** dev_ptr,
 int dlf_net_group_model(const dlf_net* net, int group, int64_t* flops, int64_t* hbm_bytes,
                         double* redundancy, int* launches);
 
-/* Name of the kernel variant that runs group g ("chain_tc", "conv_tc", "stem_tc", "conv_direct",
- * "dw3x3", "fc", "maxpool", "gavgpool"); the string is owned by the library. */
+/* Name of the kernel variant that runs group g ("chain_tc", "conv_seq", "mbconv_tc", "conv_tc", "stem_tc",
+ * "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool"); the string is owned by the library. */
 const char* dlf_net_group_kernel(const dlf_net* net, int group);
 
 /* Options (debugging and ablation); setting one clears the plan, which must be set again.
@@ -195,6 +202,11 @@ const char* dlf_net_group_kernel(const dlf_net* net, int group);
  *   DLF_OPT_SINGLE_AS_CHAIN  1: a single stride-1 1x1 / 3x3 convolution with <= 256 output
  *                               channels runs through the fused-chain kernel (input tile
  *                               loaded once) instead of the per-tap kernel.
+ *   DLF_OPT_GROUP_KERNEL     which kernel runs a multi-layer group of dense convolutions.  0 (default): narrow stride-1
+ *                               1x1 / 3x3 chains (at most 64 channels) are handed over tile by tile in shared memory, every
+ *                               other run of dense convolutions layer by layer through L2 inside one persistent kernel
+ *                               (device-wide barrier between layers); 1: shared memory wherever the chain kernel can hold
+ *                               the group; 2: L2 wherever possible.
  *   DLF_OPT_CUDA_GRAPH       1 (default): dlf_net_run replays one CUDA graph that holds every
  *                               group of the plan (captured on the first run and whenever the
  *                               input / output pointers, weights, workspace or plan change);
@@ -207,7 +219,7 @@ const char* dlf_net_group_kernel(const dlf_net* net, int group);
  *                               its three taps where that cuts the bytes a CTA streams by a fifth; 0: never (one
  *                               window load per tap); 2: wherever it applies.  Process-wide; does not clear the plan. */
 enum { DLF_OPT_NO_TENSOR_CORE = 1, /* 2 is unused */ DLF_OPT_SINGLE_AS_CHAIN = 3, DLF_OPT_CUDA_GRAPH = 4, DLF_OPT_PDL = 5,
-       DLF_OPT_CONV_ROW_MODE = 6 };
+       DLF_OPT_CONV_ROW_MODE = 6, DLF_OPT_GROUP_KERNEL = 7 };
 int dlf_net_set_option(dlf_net* net, int option, int value);
 
 /* Size of the scratch array that dlf_conv_chain_run_static keeps inside the library image. */

@@ -14,7 +14,7 @@ OK, E_INVALID_ARG, E_SHAPE, E_PLAN, E_WORKSPACE, E_UNSUPPORTED, E_CUDA, E_TIMEOU
     0, -1, -2, -3, -4, -5, -6, -7, -8)
 OPS = {"conv": 0, "dwconv": 1, "fc": 2, "maxpool": 3, "gavgpool": 4}
 ACTS = {"none": 0, "relu": 1, "relu6": 2}
-OPT_NO_TENSOR_CORE, OPT_SINGLE_AS_CHAIN, OPT_CUDA_GRAPH, OPT_PDL, OPT_CONV_ROW_MODE = 1, 3, 4, 5, 6
+OPT_NO_TENSOR_CORE, OPT_SINGLE_AS_CHAIN, OPT_CUDA_GRAPH, OPT_PDL, OPT_CONV_ROW_MODE, OPT_GROUP_KERNEL = 1, 3, 4, 5, 6, 7
 
 
 class LayerDesc(C.Structure):
@@ -64,6 +64,7 @@ def lib():
             "dlf_net_plan_unfused": (C.c_int, [vp]),
             "dlf_net_get_plan": (C.c_int, [vp, ip, i32p, i32p]),
             "dlf_net_group_is_legal": (C.c_int, [vp, C.c_int, C.c_int, C.c_int]),
+            "dlf_net_tuner_may_fuse": (C.c_int, [vp, C.c_int, C.c_int, C.c_int, C.c_int]),
             "dlf_net_autotune": (C.c_int, [vp, C.POINTER(TunerParams), ip, i32p, i32p]),
             "dlf_net_bruteforce": (C.c_int, [vp, C.POINTER(SearchParams), vp, vp, ip, i32p, i32p, fp]),
             "dlf_net_time_span": (C.c_int, [vp, C.c_int, C.c_int, C.c_int, vp, vp, C.c_int, C.c_int, C.c_int, fp]),
@@ -168,6 +169,13 @@ def net_group_is_legal(net, first, last, sm_count):
     r = lib().dlf_net_group_is_legal(net, first, last, sm_count)
     if r < 0:
         raise DlfError(r, "dlf_net_group_is_legal")
+    return bool(r)
+
+
+def net_tuner_may_fuse(net, first, last, prefix, s_max):
+    r = lib().dlf_net_tuner_may_fuse(net, first, last, 1 if prefix else 0, s_max)
+    if r < 0:
+        raise DlfError(r, "dlf_net_tuner_may_fuse")
     return bool(r)
 
 

@@ -60,8 +60,8 @@ int encode_tmap(void* out_map, const void* base, int rank, const uint64_t* dims,
     return DLF_OK;
 }
 
-enum Kind { K_CHAIN_TC, K_CONV_TC, K_CONV_DIRECT, K_DW, K_FC, K_MAXPOOL, K_GAVG, K_STEM_TC, K_MBCONV };
-static const char* kKindName[] = {"chain_tc", "conv_tc", "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool", "stem_tc", "mbconv_tc"};
+enum Kind { K_CHAIN_TC, K_CONV_TC, K_CONV_DIRECT, K_DW, K_FC, K_MAXPOOL, K_GAVG, K_STEM_TC, K_MBCONV, K_CONV_SEQ };
+static const char* kKindName[] = {"chain_tc", "conv_tc", "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool", "stem_tc", "mbconv_tc", "conv_seq"};
 
 struct Layer {
     dlf_layer_desc d;
@@ -103,7 +103,7 @@ struct dlf_net {
     uint8_t* ws = nullptr;
     size_t ws_bytes = 0, ws_need = 0, in_off = 0, in_bytes = 0, status_off = 0, splitk_off = 0;
     int dev_sms = 0;
-    int opt_no_tc = 0, opt_single_chain = 0, opt_graph = 1;
+    int opt_no_tc = 0, opt_single_chain = 0, opt_graph = 1, opt_group_kernel = 0;
     const void* last_out = nullptr;
     // One CUDA graph per (input, output) pointer pair holds the whole plan; a second, instrumented
     // one records an event after every group for per-group timing.
@@ -141,24 +141,8 @@ static bool chain_layer_ok(const Layer& l) {
            d.pad == d.kh / 2 && chain_tc_layer_supported(d.cin, d.cout, d.kh);
 }
 
-// A fused group re-streams each layer's weights for every tile, so a layer may join other layers
-// only while its weights stay small next to the tile it works on.
-constexpr int64_t kMaxFusedWeightBytes = 160 * 1024;
-
-// The tuner (max_layer_flops > 0) also keeps a layer with more work than that out of multi-layer chains: the fused
-// kernel runs a tile's layers one after the other and recomputes halos, which pays only for layers that are short
-// (Sec. IV-B of the paper finds the same: fusion helps its 0.43 G-operation layer and hurts its 1.72 G-operation
-// one).  Measured here: 1x1 64->64 + 3x3 64->64 at 56x56, batch 32 takes 37 us fused, 31 us as two kernels.
-// A plan given explicitly may still ask for such a chain.
-static const double kTunerMaxFusedFlopsPerSm = 2.0e7;
-
-static bool span_is_chain(const dlf_net* net, int first, int last, double max_layer_flops = 0.0) {
+static bool span_is_chain(const dlf_net* net, int first, int last) {
     if (last - first + 1 > kMaxChain) return false;
-    if (last > first)
-        for (int i = first; i <= last; i++) {
-            if (net->layers[i].w_elems * 2 > kMaxFusedWeightBytes) return false;
-            if (max_layer_flops > 0.0 && static_cast<double>(net->layers[i].flops) > max_layer_flops) return false;
-        }
     const int n = static_cast<int>(net->layers.size());
     for (int i = first; i <= last; i++) {
         const Layer& l = net->layers[i];
@@ -333,6 +317,21 @@ static ConvArgs fc_as_conv_args(const dlf_net* net, int i, const void* in_dev, v
     return a;
 }
 
+// ---- groups handed over through L2 -------------------------------------------------------------------------------------
+// Any run of dense convolutions the single-layer tensor-core kernel takes (any kernel size, stride 1 or 2, fused pool,
+// residual from anywhere, a projection branch) can run as ONE persistent kernel whose CTAs walk the layers together with a
+// device-wide barrier in between; every layer's map goes to its workspace slot.
+static bool span_is_seq(const dlf_net* net, int first, int last) {
+    if (net->opt_no_tc || last - first + 1 > conv_seq_max_layers()) return false;
+    for (int i = first; i <= last; i++) {
+        const Layer& l = net->layers[i];
+        if (l.d.op != DLF_CONV || l.d.groups != 1) return false;
+        ConvArgs a = conv_args(net, i, nullptr, nullptr);
+        if (!conv_seq_layer_supported(a)) return false;
+    }
+    return true;
+}
+
 static bool single_kind(const dlf_net* net, int i, Kind* kind) {
     const Layer& l = net->layers[i];
     switch (l.d.op) {
@@ -385,12 +384,53 @@ static bool make_group(const dlf_net* net, int first, int last, int sms, Group* 
         g->kind = K_MBCONV;
         return g->mb_tiling.ok;
     }
+    // Two ways to fuse dense convolutions: hand-over in shared memory (a chain of stride-1 1x1 / 3x3 layers, tile by tile) or
+    // through L2 (any run of dense convolutions, layer by layer behind a device-wide barrier).  Unless an option says
+    // otherwise the first is taken for narrow layers (at most 64 channels: there it was measured faster), the second elsewhere.
+    const bool chain_ok = span_is_chain(net, first, last);
+    const bool seq_ok = first < last && span_is_seq(net, first, last);
+    bool narrow = true;
+    for (int i = first; i <= last; i++) narrow = narrow && net->layers[i].d.cin <= 64 && net->layers[i].d.cout <= 64;
+    const bool want_chain = chain_ok && (first == last || net->opt_group_kernel == 1 || (net->opt_group_kernel == 0 && narrow) || !seq_ok);
+    if (want_chain) {
+        ChainArgs a = chain_args(net, first, last, nullptr, nullptr);
+        g->tiling = chain_tc_tiling(a, sms, net->dev_sms);
+        g->kind = K_CHAIN_TC;
+        if (g->tiling.ok) return true;
+        if (first == last) return single_kind(net, first, &g->kind);
+    }
+    if (seq_ok) {
+        g->kind = K_CONV_SEQ;
+        return true;
+    }
+    return false;
+}
+
+// ---- what the tuner may propose as one group --------------------------------------------------------------------
+// Algorithm 1 grows a block while the layers can run as one kernel AND that kernel is expected to pay (Sec. IV-B: fusing
+// helps layers with few operations and hurts heavy ones).  For a dense chain the estimate is the fused kernel's own cost
+// model (the tiler's SM clocks at 1.9 GHz) against one kernel per layer: the slower of a layer's operations at 600 TFLOP/s
+// and its bytes at 5.5 TB/s (what the single-layer kernel reaches on this chip) plus 5.5 us per kernel boundary.
+// Inverted-residual blocks follow the measured rule on the hidden width.  Groups handed over through L2 are proposed only
+// when the option asks for them (measured: a device-wide barrier per layer is no cheaper than a kernel boundary).
+// `prefix`: the layers may also be the beginning of a pattern that can still grow into a group.
+static bool tuner_may_fuse(const dlf_net* net, int first, int last, bool prefix, int s_max) {
+    if (first == last) return true;
+    if (net->opt_no_tc) return false;
+    if (span_is_mbconv(net, first, last, prefix, kTunerMaxHidden)) return true;
+    if (net->opt_group_kernel == 2 && span_is_seq(net, first, last)) return true;
     if (!span_is_chain(net, first, last)) return false;
-    ChainArgs a = chain_args(net, first, last, nullptr, nullptr);
-    g->tiling = chain_tc_tiling(a, sms, net->dev_sms);
-    g->kind = K_CHAIN_TC;
-    if (!g->tiling.ok && first == last) return single_kind(net, first, &g->kind);
-    return g->tiling.ok;
+    if (net->opt_group_kernel == 1) return true;
+    const ChainTiling t = chain_tc_tiling(chain_args(net, first, last, nullptr, nullptr), s_max, s_max);
+    if (!t.ok) return false;
+    double single_us = 0.0;
+    for (int i = first; i <= last; i++) {
+        const Layer& l = net->layers[i];
+        const double bytes = static_cast<double>(l.in[0] * l.in[1] * l.in[2] * l.in[3] * 2) + static_cast<double>(l.bytes) + static_cast<double>(l.w_elems * 2) +
+                             (l.d.res_src != -2 ? static_cast<double>(l.bytes) : 0.0);
+        single_us += std::max(static_cast<double>(l.flops) / 600e6, bytes / 5.5e6) + 5.5;
+    }
+    return t.cost / 1.9e3 < single_us;
 }
 
 static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* final_out, cudaStream_t s) {
@@ -402,6 +442,14 @@ static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* 
         case K_CHAIN_TC: {
             ChainArgs a = chain_args(net, g.first, g.last, in_dev, y);
             return launch_chain_tc(a, g.tiling, g.sms, status, s);
+        }
+        case K_CONV_SEQ: {
+            ConvArgs a[16];
+            const int cnt = g.last - g.first + 1;
+            if (cnt > 16) return DLF_E_PLAN;
+            for (int i = g.first; i <= g.last; i++)
+                a[i - g.first] = conv_args(net, i, in_dev, i == n - 1 ? final_out : static_cast<void*>(net->ws + net->layers[i].off));
+            return launch_conv_seq(a, cnt, g.sms, status, reinterpret_cast<unsigned*>(status) + 2, s);
         }
         case K_MBCONV: return launch_mbconv_tc(mbconv_args(net, g.first, g.last, in_dev, y), g.mb_tiling, g.sms, status, s);
         case K_CONV_TC:
@@ -517,18 +565,24 @@ static int validate_plan(const dlf_net* net, int n_groups, const int32_t* ends, 
         is_end[prev] = 1;
     }
     if (prev != n - 1) return DLF_E_PLAN;
-    // a tensor read across a group boundary must have reached HBM
     int first = 0;
     out->clear();
+    std::vector<char> stored(n, 0);   // the layer's map reaches its workspace slot: a group's last layer, any layer of an L2 group
+    for (int g = 0; g < n_groups; g++) {
+        Group grp;
+        if (!make_group(net, first, ends[g], sms[g], &grp)) return DLF_E_PLAN;
+        out->push_back(grp);
+        for (int i = first; i <= ends[g]; i++) stored[i] = (i == ends[g] || grp.kind == K_CONV_SEQ) ? 1 : 0;
+        first = ends[g] + 1;
+    }
+    // a tensor read across a group boundary must have been stored
+    first = 0;
     for (int g = 0; g < n_groups; g++) {
         for (int i = first; i <= ends[g]; i++) {
             const int refs[2] = {net->layers[i].d.src, net->layers[i].d.res_src};
             for (int r : refs)
-                if (r >= 0 && r < first && !is_end[r]) return DLF_E_PLAN;
+                if (r >= 0 && r < first && !stored[r]) return DLF_E_PLAN;
         }
-        Group grp;
-        if (!make_group(net, first, ends[g], sms[g], &grp)) return DLF_E_PLAN;
-        out->push_back(grp);
         first = ends[g] + 1;
     }
     return DLF_OK;
@@ -754,6 +808,11 @@ int dlf_net_group_is_legal(const dlf_net* net, int first, int last, int sm_count
     return make_group(net, first, last, sm_count, &g) ? 1 : 0;
 }
 
+int dlf_net_tuner_may_fuse(const dlf_net* net, int first, int last, int prefix, int s_max) {
+    if (!net || first < 0 || last < first || last >= static_cast<int>(net->layers.size()) || s_max < 1) return DLF_E_INVALID_ARG;
+    return tuner_may_fuse(net, first, last, prefix != 0, s_max) ? 1 : 0;
+}
+
 int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_groups, int32_t* group_end,
                      int32_t* sm_count) {
     if (!net || !params || !n_groups || !group_end || !sm_count) return DLF_E_INVALID_ARG;
@@ -771,7 +830,6 @@ int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_
     const int n = static_cast<int>(net->layers.size());
     double sum_op = 0.0, sum_mp = 0.0;
     int block = 0, start = 0, ng = 0;
-    const double max_fl = kTunerMaxFusedFlopsPerSm * s_max;
     for (int i = 0; i < n; i++) {
         const Layer& l = net->layers[i];
         if (is_param(l)) {
@@ -781,11 +839,11 @@ int dlf_net_autotune(const dlf_net* net, const dlf_tuner_params* params, int* n_
         }
         // a block may grow while its layers are, or can still become, a group one kernel runs; it may
         // close only where they already are one (inside an inverted-residual block it keeps growing)
-        bool forced = (i == n - 1) || !(span_is_chain(net, start, i + 1, max_fl) || span_is_mbconv(net, start, i + 1, true, kTunerMaxHidden));
-        const bool closable = (i == start) || span_is_chain(net, start, i, max_fl) || span_is_mbconv(net, start, i, false, kTunerMaxHidden);
+        bool forced = (i == n - 1) || !tuner_may_fuse(net, start, i + 1, true, s_max);
+        const bool closable = (i == start) || tuner_may_fuse(net, start, i, false, s_max);
         if (!forced && params->legalise) {
             Group g;
-            if (i + 1 > start && (span_is_chain(net, start, i + 1, max_fl) || span_is_mbconv(net, start, i + 1, false, kTunerMaxHidden)))
+            if (i + 1 > start && tuner_may_fuse(net, start, i + 1, false, s_max))
                 forced = !make_group(net, start, i + 1, s_max, &g);
         }
         if (block > 0) {
@@ -846,7 +904,7 @@ int dlf_net_sync(dlf_net* net, void* stream) {
         if (e != cudaSuccess) return cuda_fail(e);
         if (st != 0) {
             g_last_cuda_error = st;
-            cudaMemset(net->ws + net->status_off, 0, sizeof(int));
+            cudaMemset(net->ws + net->status_off, 0, 4 * sizeof(int));   // the status word and the multi-layer kernels' barrier counters
             // a launch that gave up may have left split-K arrival counters behind
             cudaMemset(net->ws + net->splitk_off, 0, kSplitKCounterBytes);
             return DLF_E_TIMEOUT;
@@ -1084,6 +1142,12 @@ int dlf_net_group_model(const dlf_net* net, int group, int64_t* flops, int64_t* 
         fl += l.flops;
         by += l.w_elems * 2 + (is_param(l) ? l.d.cout * 4 : 0);
         if (l.d.res_src != -2 && l.d.res_src < g.first) by += l.out[0] * l.ho_pre * l.wo_pre * l.out[3] * 2;
+        // a group handed over through L2 still writes every map to its slot and reads it back: counted like separate layers
+        if (g.kind == K_CONV_SEQ) {
+            if (i > g.first) by += l.in[0] * l.in[1] * l.in[2] * l.in[3] * 2;
+            if (i < g.last) by += static_cast<int64_t>(l.bytes);
+            if (l.d.res_src != -2 && l.d.res_src >= g.first) by += l.out[0] * l.ho_pre * l.wo_pre * l.out[3] * 2;
+        }
     }
     if (flops) *flops = fl;
     if (hbm_bytes) *hbm_bytes = by;
@@ -1102,6 +1166,10 @@ int dlf_net_set_option(dlf_net* net, int option, int value) {
     switch (option) {
         case DLF_OPT_NO_TENSOR_CORE: net->opt_no_tc = value != 0; break;
         case DLF_OPT_SINGLE_AS_CHAIN: net->opt_single_chain = value != 0; break;
+        case DLF_OPT_GROUP_KERNEL:
+            if (value < 0 || value > 2) return DLF_E_INVALID_ARG;
+            net->opt_group_kernel = value;
+            break;
         case DLF_OPT_CUDA_GRAPH: net->opt_graph = value != 0; return DLF_OK;
         case DLF_OPT_PDL: g_use_pdl = value != 0; invalidate_graphs(net); return DLF_OK;
         case DLF_OPT_CONV_ROW_MODE:

@@ -34,6 +34,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstring>
 
 #include "internal.h"
 #include "ptx.cuh"
@@ -99,56 +100,62 @@ __device__ __forceinline__ TileCoord decode_work(const ConvTcParams& p, int t) {
     return c;
 }
 
-template <int ACT, bool POOL, bool RES, bool ROW, bool SPLIT>
-__global__ void __launch_bounds__(kThreads, 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
-               const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmr, const ConvTcParams p) {
-    extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[8], empty_bar[8], tfull_bar[2], tempty_bar[2];
-    __shared__ uint64_t sfull_bar[2], sfree_bar[2];  // staging buffer: filled by the epilogue / free again (residual landed)
-    __shared__ uint32_t tmem_base_s;
-    __shared__ int abort_s;
+// Device-wide barrier of a multi-layer launch (all CTAs resident, one per SM): every CTA adds one to a counter in global
+// memory when it has finished a layer; a warp that is about to read what another CTA wrote in an earlier layer of the same
+// launch first waits until the counter has reached `target` = layers finished x CTAs.  Bounded like every other wait.
+struct GridSync {
+    unsigned* counter;   // null: a single-layer launch, nothing to wait for
+    unsigned target;
+};
+__device__ __forceinline__ bool grid_wait(const GridSync& gs, int lane, volatile int* abort_flag, int* status) {
+    if (gs.counter == nullptr || gs.target == 0u) return true;
+    bool ok = true;
+    if (lane == 0) {
+        uint64_t t0 = 0;
+        uint32_t spins = 0;
+        while (true) {
+            unsigned v;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(gs.counter) : "memory");
+            if (v >= gs.target) break;
+            if (spins > 8) __nanosleep(64);
+            if ((++spins & 63u) == 0) {
+                if (*abort_flag) { ok = false; break; }
+                const uint64_t now = global_ns();
+                if (t0 == 0) t0 = now;
+                if (now - t0 > kWaitLimitNs) {
+                    *abort_flag = 1;
+                    atomicCAS(status, 0, 0x700 | (blockIdx.x << 12));
+                    ok = false;
+                    break;
+                }
+            }
+        }
+        __threadfence();
+        if (gs.target == gridDim.x && threadIdx.x == 32 * kProdWarp0) DLF_TRACE_POINT(status, 27);
+    }
+    ok = __all_sync(0xffffffffu, ok);
+    // what the other CTAs stored (TMA stores) is read here through the async proxy (TMA loads) as well
+    asm volatile("fence.proxy.async;" ::: "memory");
+    return ok;
+}
 
-    if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 0);
-    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t* stage0 = smem_raw + (base - smem_u32(smem_raw));
+// The barriers of one CTA (static shared memory of the kernel that calls the roles).
+struct ConvBars {
+    uint64_t *full_bar, *empty_bar, *tfull_bar, *tempty_bar, *sfull_bar, *sfree_bar;
+    int* abort_s;
+};
+
+// The warp roles of one layer: everything between the CTA's set-up (barriers initialised, tensor memory allocated) and
+// its wind-down.  Called once by the single-layer kernel and once per layer by the multi-layer kernel.
+template <int ACT, bool POOL, bool RES, bool ROW, bool SPLIT>
+__device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CUtensorMap* tmw_p, const CUtensorMap* tmy_p,
+                                              const CUtensorMap* tmr_p, const ConvTcParams& p, const ConvBars& sm, uint32_t tmem_base,
+                                              uint8_t* stage0, uint32_t base, const GridSync& gs) {
     float* bias_s = reinterpret_cast<float*>(stage0 + p.bias_off);
     constexpr int kTps = ROW ? 3 : 1;   // taps per ring stage: a whole kernel row in the row mode
     const int stage_bytes = p.kg * (p.a_bytes + kTps * p.BN * 128);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    volatile int* abort_flag = &abort_s;
-
-    if (threadIdx.x == 0) {
-        abort_s = 0;
-        for (int i = 0; i < p.stages; i++) {
-            mbar_init(&full_bar[i], 2);  // the A and the B producer each arrive with their byte count
-            mbar_init(&empty_bar[i], 1);
-        }
-        for (int i = 0; i < 2; i++) {
-            mbar_init(&tfull_bar[i], 1);
-            mbar_init(&tempty_bar[i], kEpiWarps);
-            mbar_init(&sfull_bar[i], kEpiWarps);
-            mbar_init(&sfree_bar[i], 1);
-        }
-        fence_barrier_init();
-        tma_prefetch_desc(&tmx);
-        tma_prefetch_desc(&tmw);
-        if (!POOL) tma_prefetch_desc(&tmy);
-        if (!POOL && RES) tma_prefetch_desc(&tmr);
-    }
-    if (warp == kMmaWarp) {
-        tmem_alloc(&tmem_base_s, p.tmem_cols);
-        tmem_relinquish();
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    pdl_launch_dependents();
-    // everything above overlapped the previous kernel; from here on its outputs are read - except by the
-    // weight producers, which only read constants and may run ahead
-    if (warp < kProdWarp0 + 2 || warp == kStoreWarp) pdl_wait();
-    if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
-    const uint32_t tmem_base = tmem_base_s;
+    volatile int* abort_flag = sm.abort_s;
     const int k_iters = p.tgroups * p.kgroups;
 
     if (warp == kStoreWarp) {
@@ -156,28 +163,31 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         // One lane per 64-channel plane: a thread's bulk copies run one after the other (about 0.3 us each,
         // measured), the copies of different lanes side by side.
         if (!POOL && !SPLIT) {   // (split-K tiles leave through the partial sums in global memory)
+            if (RES && !grid_wait(gs, lane, abort_flag, p.status)) return;   // the residual may be a layer of this launch
             uint8_t* stage_out = stage0 + p.stage_out_off;
             auto planes_of = [&](const TileCoord& c) { return (min(p.BN, ((p.Cout - c.co0) + 15) & ~15) + 63) >> 6; };
             auto fetch_residual = [&](int t, uint32_t b) {
                 const TileCoord c = decode_work(p, t);
                 const int planes = planes_of(c);
-                if (lane == 0) mbar_expect_tx(&sfree_bar[b], static_cast<uint32_t>(planes * p.rows) * 128u);
+                if (lane == 0) mbar_expect_tx(&sm.sfree_bar[b], static_cast<uint32_t>(planes * p.rows) * 128u);
                 __syncwarp();
                 if (lane < planes)
-                    tma_load_4d(stage_out + b * p.out_buf_bytes + lane * kABytes, &tmr, &sfree_bar[b], c.co0 + lane * 64, c.wo0, c.ho0, c.n0);
+                    tma_load_4d(stage_out + b * p.out_buf_bytes + lane * kABytes, tmr_p, &sm.sfree_bar[b], c.co0 + lane * 64, c.wo0, c.ho0, c.n0);
             };
             if (RES)
+#pragma unroll 1
                 for (int jj = 0; jj < p.out_bufs; jj++)
                     if (static_cast<int>(blockIdx.x) + jj * static_cast<int>(gridDim.x) < p.n_work) fetch_residual(blockIdx.x + jj * gridDim.x, jj);
             uint32_t j = 0;
             DLF_TRACE_DECL(sacc, smark);  // cycles of CTA 0's store warp: 0 wait for a staged tile, 1 store and its read, 2 residual fetch
+#pragma unroll 1
             for (int t = blockIdx.x; t < p.n_work; t += gridDim.x, j++) {
                 const uint32_t b = j % p.out_bufs, ph = (j / p.out_bufs) & 1u;
-                if (!mbar_wait_warp(&sfull_bar[b], ph, abort_flag, p.status, 0x500 | (blockIdx.x << 12))) break;
+                if (!mbar_wait_warp(&sm.sfull_bar[b], ph, abort_flag, p.status, 0x500 | (blockIdx.x << 12))) break;
                 DLF_TRACE_ACC(sacc, 0, smark);
                 const TileCoord c = decode_work(p, t);
                 if (lane < planes_of(c)) {
-                    tma_store_4d(&tmy, stage_out + b * p.out_buf_bytes + lane * kABytes, c.co0 + lane * 64, c.wo0, c.ho0, c.n0);
+                    tma_store_4d(tmy_p, stage_out + b * p.out_buf_bytes + lane * kABytes, c.co0 + lane * 64, c.wo0, c.ho0, c.n0);
                     tma_store_commit();
                     tma_store_wait_read();  // the plane has been read: it may take the next residual / the next tile
                 }
@@ -187,7 +197,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 if (RES) {
                     if (t2 < p.n_work) fetch_residual(t2, b);
                 } else if (lane == 0) {
-                    mbar_arrive(&sfree_bar[b]);
+                    mbar_arrive(&sm.sfree_bar[b]);
                 }
                 DLF_TRACE_ACC(sacc, 2, smark);
             }
@@ -202,6 +212,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         {
             const int role = warp - kProdWarp0;
             const bool is_b = role >= 2;
+            if (!is_b && !grid_wait(gs, lane, abort_flag, p.status)) return;   // the input may be a layer of this launch
             const uint32_t parity = role & 1;
             const uint32_t my_bytes = static_cast<uint32_t>(p.kg) * (is_b ? static_cast<uint32_t>(kTps * p.BN) : static_cast<uint32_t>(p.rows)) * 128u;
             uint32_t it = 0;
@@ -214,24 +225,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 // a ring stage belongs to ONE producer warp of each kind: a warp that skipped a phase of
                 // a stage's barrier could not tell "two phases ago" from "now" by parity
                 if ((st & 1u) != parity) return true;
-                if (!mbar_wait_warp(&empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status, 0x100 | (blockIdx.x << 12))) return false;
+                if (!mbar_wait_warp(&sm.empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status, 0x100 | (blockIdx.x << 12))) return false;
                 DLF_TRACE_ACC(pacc, 0, pmark);
                 const int tap = tg * kTps;
                 const int r = tap / p.kw, s = tap % p.kw;
                 uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
-                if (lane == 0) mbar_expect_tx(&full_bar[st], my_bytes);
+                if (lane == 0) mbar_expect_tx(&sm.full_bar[st], my_bytes);
                 __syncwarp();
                 if (lane < p.kg) {   // a chunk past C_in / 64 lies outside the tensor map and arrives as zeros
                     const int kc = kq * p.kg + lane;
                     if (is_b) {
                         uint8_t* dst = sa + p.kg * p.a_bytes + lane * kTps * p.BN * 128;
-                        if (p.grouped) tma_load_4d(dst, &tmw, &full_bar[st], 0, c.co0, tap, kc);
-                        else tma_load_3d(dst, &tmw, &full_bar[st], kc * 64, tap, c.co0);
+                        if (p.grouped) tma_load_4d(dst, tmw_p, &sm.full_bar[st], 0, c.co0, tap, kc);
+                        else tma_load_3d(dst, tmw_p, &sm.full_bar[st], kc * 64, tap, c.co0);
                     } else {
                         const int wi = c.wo0 * p.stride - p.pad + s, hi = c.ho0 * p.stride - p.pad + r;
                         uint8_t* dst = sa + lane * p.a_bytes;
-                        if (p.grouped) tma_load_5d(dst, &tmx, &full_bar[st], 0, wi, hi, c.n0, kc);
-                        else tma_load_4d(dst, &tmx, &full_bar[st], kc * 64, wi, hi, c.n0);
+                        if (p.grouped) tma_load_5d(dst, tmx_p, &sm.full_bar[st], 0, wi, hi, c.n0, kc);
+                        else tma_load_4d(dst, tmx_p, &sm.full_bar[st], kc * 64, wi, hi, c.n0);
                     }
                 }
                 __syncwarp();
@@ -239,13 +250,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 DLF_TRACE_ACC(pacc, 1, pmark);
                 return true;
             };
+#pragma unroll 1
             for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x) {
                 const TileCoord c = decode_work<SPLIT>(p, t);
                 if (SPLIT) {   // this item's share of the tile's (tap group, K-chunk group) list
                     const int l0 = c.ks * p.kgs, l1 = min(k_iters, l0 + p.kgs);
+#pragma unroll 1
                     for (int li = l0; li < l1 && ok; li++, it++) ok = load_stage(c, li / p.kgroups, li % p.kgroups);
                 } else {
+#pragma unroll 1
                     for (int tg = 0; tg < p.tgroups && ok; tg++)
+#pragma unroll 1
                         for (int kq = 0; kq < p.kgroups && ok; kq++, it++) ok = load_stage(c, tg, kq);
                 }
             }
@@ -260,9 +275,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         uint32_t it = 0, j = 0;
         bool ok = true;
         DLF_TRACE_DECL(macc, mmark);  // cycles of CTA 0's issuer: 0 accumulator wait, 1 stage wait, 2 issue
+#pragma unroll 1
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
             const uint32_t acc = j & 1u;
-            ok = mbar_wait_warp(&tempty_bar[acc], ((j >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x200 | (blockIdx.x << 12));
+            ok = mbar_wait_warp(&sm.tempty_bar[acc], ((j >> 1) & 1u) ^ 1u, abort_flag, p.status, 0x200 | (blockIdx.x << 12));
             if (!ok) break;
             DLF_TRACE_ACC(macc, 0, mmark);
             tc_fence_after_sync();
@@ -273,9 +289,10 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 k_end = min(k_iters - l0, p.kgs);
                 kq = l0 % p.kgroups;
             }
+#pragma unroll 1
             for (int ki = 0; ki < k_end; ki++, it++) {
                 const int st = it % p.stages;
-                ok = mbar_wait_warp(&full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
+                ok = mbar_wait_warp(&sm.full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                 if (!ok) break;
                 if (it == 0 && lane == 0) DLF_TRACE_POINT(p.status, 3);
                 DLF_TRACE_ACC(macc, 1, mmark);
@@ -285,6 +302,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 const int g_end = min(p.kg, p.kchunks - kq * p.kg);
                 if (elect_one()) {
                     if (!ROW) {
+#pragma unroll 1
                         for (int g = 0; g < g_end; g++) {
                             const uint64_t ad = a0 + static_cast<uint32_t>(g) * a_chunk16, bd = b0 + static_cast<uint32_t>(g) * b_chunk16;
                             const int ksteps = (kq * p.kg + g == p.kchunks - 1) ? p.ksteps_last : 4;
@@ -296,6 +314,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     } else {
                         // row mode (whole 64-channel chunks): the three taps of a kernel row read the same window, one
                         // pixel (one 128-byte row) further each
+#pragma unroll 1
                         for (int g = 0; g < g_end; g++) {
                             uint64_t ad = a0 + static_cast<uint32_t>(g) * a_chunk16, bd = b0 + static_cast<uint32_t>(g * 3) * b_chunk16;
 #pragma unroll
@@ -307,13 +326,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                             }
                         }
                     }
-                    umma_commit(&empty_bar[st]);  // frees the stage once these MMAs have read it
+                    umma_commit(&sm.empty_bar[st]);  // frees the stage once these MMAs have read it
                 }
                 __syncwarp();
                 DLF_TRACE_ACC(macc, 2, mmark);
                 if (++kq == p.kgroups) kq = 0;
             }
-            if (ok && elect_one()) umma_commit(&tfull_bar[acc]);
+            if (ok && elect_one()) umma_commit(&sm.tfull_bar[acc]);
             __syncwarp();
             if (j == 0 && lane == 0) DLF_TRACE_POINT(p.status, 4);
         }
@@ -330,12 +349,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         {   // bias of every output channel, zero past C_out (the channel tile is padded to 16): staged by the epilogue
             // warps alone, after the CTA-wide barrier, so that the producers' first copies do not wait for these loads
             const int n_bias = p.n_tiles_n * p.BN;
+#pragma unroll 1
             for (int i = threadIdx.x; i < n_bias; i += 32 * kEpiWarps) bias_s[i] = i < p.Cout ? __ldg(p.bias + i) : 0.0f;
             asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
         }
         uint32_t j = 0;
         bool ok = true;
+        if (RES && POOL) ok = grid_wait(gs, lane, abort_flag, p.status);   // residual read with plain loads
         DLF_TRACE_DECL(eacc, emark);  // cycles of CTA 0's first epilogue thread: 0 staging-buffer wait, 1 accumulator wait, 2 drain
+#pragma unroll 1
         for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x, j++) {
             const TileCoord c = decode_work<SPLIT>(p, t);
             const uint32_t acc = j & 1u;
@@ -349,12 +371,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 // Split-K: this item's raw fp32 sums go to global memory; of the items of one tile, the warp that
                 // arrives last at the (tile, warp) counter adds the shares up in their fixed order (so the result
                 // does not depend on which was last), applies bias and activation and writes the fp16 output.
-                ok = mbar_wait(&tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
+                ok = mbar_wait(&sm.tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
                 if (!ok) break;
                 tc_fence_after_sync();
                 const uint32_t taddr = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * p.acc_stride;
                 const size_t share = static_cast<size_t>(p.rows) * p.acc_stride;   // floats of one item's partial tile
                 float* tile0 = p.partial + static_cast<size_t>(c.tile) * p.splits * share + static_cast<size_t>(min(m, p.rows - 1)) * p.acc_stride;
+#pragma unroll 1
                 for (int cc = part * 32; cc < ncols; cc += 32 * kEpiParts) {
                     uint32_t r[32];
                     __syncwarp();
@@ -369,7 +392,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 }
                 tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&tempty_bar[acc]);
+                if (lane == 0) mbar_arrive(&sm.tempty_bar[acc]);
                 __threadfence();
                 __syncwarp();
                 int* cnt = p.counters + c.tile * kEpiWarps + warp;
@@ -379,6 +402,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                 if (old == p.splits - 1) {
                     __threadfence();
                     if (valid) {
+#pragma unroll 1
                         for (int cc = part * 32; cc < ncols; cc += 32 * kEpiParts) {
                             const int nc = min(32, ncols - cc);
 #pragma unroll
@@ -389,6 +413,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                                 const float4 b1 = *reinterpret_cast<const float4*>(bias_s + co + 4);
                                 float a[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
                                 const float4* src = reinterpret_cast<const float4*>(tile0 + cc + g * 8);
+#pragma unroll 1
                                 for (int sp = 0; sp < p.splits; sp++, src += share / 4) {
                                     const float4 v0 = __ldcg(src), v1 = __ldcg(src + 1);
                                     a[0] += v0.x; a[1] += v0.y; a[2] += v0.z; a[3] += v0.w;
@@ -429,11 +454,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             uint8_t* sout = stage_out + (j % p.out_bufs) * p.out_buf_bytes;
             if (!POOL) {   // the staging buffer is free (first uses pass at once) / holds this tile's residual
                 const uint32_t ph = (j / p.out_bufs) & 1u;
-                ok = mbar_wait(&sfree_bar[j % p.out_bufs], RES ? ph : ph ^ 1u, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
+                ok = mbar_wait(&sm.sfree_bar[j % p.out_bufs], RES ? ph : ph ^ 1u, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
                 if (!ok) break;
             }
             DLF_TRACE_ACC(eacc, 0, emark);
-            ok = mbar_wait(&tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
+            ok = mbar_wait(&sm.tfull_bar[acc], (j >> 1) & 1u, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
             if (!ok) break;
             DLF_TRACE_ACC(eacc, 1, emark);
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 5);
@@ -497,6 +522,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                     rok = rok_next;
                 }
             };
+#pragma unroll 1
             for (int cc = part * 32; cc < ncols; cc += 32 * kEpiParts) {
                 uint32_t r[32];
                 __syncwarp();  // the aligned TMEM load needs the whole warp converged
@@ -506,17 +532,78 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
             }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&tempty_bar[acc]);  // the accumulator is drained
+            if (lane == 0) mbar_arrive(&sm.tempty_bar[acc]);  // the accumulator is drained
             if (!POOL) {
                 fence_proxy_async_smem();  // the staging tile is read by the TMA unit
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sfull_bar[j % p.out_bufs]);
+                if (lane == 0) mbar_arrive(&sm.sfull_bar[j % p.out_bufs]);
             }
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 6);
             DLF_TRACE_ACC(eacc, 2, emark);
         }
         if (issuer) DLF_TRACE_FLUSH_N(p.status, eacc, 8, 3);
     }
+
+}
+
+// Initialises the barriers for a ring of `stages` stages (thread 0; `again`: they hold valid objects already).
+__device__ __forceinline__ void conv_tc_init_bars(const ConvBars& sm, int stages, bool again) {
+    if (again) {
+        for (int i = 0; i < 8; i++) { mbar_inval(&sm.full_bar[i]); mbar_inval(&sm.empty_bar[i]); }
+        for (int i = 0; i < 2; i++) { mbar_inval(&sm.tfull_bar[i]); mbar_inval(&sm.tempty_bar[i]); mbar_inval(&sm.sfull_bar[i]); mbar_inval(&sm.sfree_bar[i]); }
+    }
+    for (int i = 0; i < (again ? 8 : stages); i++) {
+        mbar_init(&sm.full_bar[i], 2);  // the A and the B producer each arrive with their byte count
+        mbar_init(&sm.empty_bar[i], 1);
+    }
+    for (int i = 0; i < 2; i++) {
+        mbar_init(&sm.tfull_bar[i], 1);
+        mbar_init(&sm.tempty_bar[i], kEpiWarps);
+        mbar_init(&sm.sfull_bar[i], kEpiWarps);
+        mbar_init(&sm.sfree_bar[i], 1);
+    }
+    fence_barrier_init();
+}
+
+template <int ACT, bool POOL, bool RES, bool ROW, bool SPLIT>
+__global__ void __launch_bounds__(kThreads, 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
+               const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmr, const ConvTcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[8], empty_bar[8], tfull_bar[2], tempty_bar[2];
+    __shared__ uint64_t sfull_bar[2], sfree_bar[2];  // staging buffer: filled by the epilogue / free again (residual landed)
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+
+    if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 0);
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* stage0 = smem_raw + (base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const ConvBars sm{full_bar, empty_bar, tfull_bar, tempty_bar, sfull_bar, sfree_bar, &abort_s};
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        conv_tc_init_bars(sm, p.stages, false);
+        tma_prefetch_desc(&tmx);
+        tma_prefetch_desc(&tmw);
+        if (!POOL) tma_prefetch_desc(&tmy);
+        if (!POOL && RES) tma_prefetch_desc(&tmr);
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(&tmem_base_s, p.tmem_cols);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    pdl_launch_dependents();
+    // everything above overlapped the previous kernel; from here on its outputs are read - except by the
+    // weight producers, which only read constants and may run ahead
+    if (warp < kProdWarp0 + 2 || warp == kStoreWarp) pdl_wait();
+    if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
+    const uint32_t tmem_base = tmem_base_s;
+
+    conv_tc_roles<ACT, POOL, RES, ROW, SPLIT>(&tmx, &tmw, &tmy, &tmr, p, sm, tmem_base, stage0, base, GridSync{nullptr, 0u});
 
     tc_fence_before_sync();
     __syncthreads();
@@ -525,6 +612,124 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, p.tmem_cols);
         if (lane == 0) DLF_TRACE_POINT(p.status, 7);
+    }
+}
+
+// ---- several layers in one launch ------------------------------------------------------------------------------------------
+// A fusion group of dense convolutions whose maps are too large (or whose shapes are too irregular: strides, a projection
+// branch, a residual from inside the group) to be handed over in shared memory runs as ONE persistent kernel all the same:
+// the CTAs walk the group's layers together, separated by a device-wide barrier, and a layer's output goes to its
+// workspace slot, which at these sizes stays in the 126 MB L2 until the next layer has read it.  What the group saves
+// against one kernel per layer is the kernel boundary (tear-down, launch, set-up, first descriptor fetch: about 5.5 us
+// measured, against about 2.5 us for the barrier and the first loads behind it) - the paper's "layers compiled as one block
+// on one core count" (Sec. III-B, Sec. IV-C) in the form this chip's cache makes possible.
+constexpr int kMaxSeq = 16;
+struct SeqLayer {
+    CUtensorMap tmx, tmw, tmy, tmr;
+    ConvTcParams p;
+    int variant;   // ((act * 2 + pool) * 2 + res) * 2 + row
+    int pad_[3];
+};
+struct SeqParams {
+    SeqLayer L[kMaxSeq];
+    int n_layers;
+    unsigned* sync;   // two words, zero between launches: layers finished x CTAs, CTAs done
+    int* status;
+};
+
+// One layer of a multi-layer launch, as a function of its own: each variant then gets its own register allocation
+// instead of the union of all of them inside the calling kernel.
+template <int ACT, bool POOL, bool RES, bool ROW>
+__device__ __noinline__ void conv_seq_layer(const SeqLayer* Y, const ConvTcParams* p, const ConvBars* sm, uint32_t tmem_base, uint8_t* stage0,
+                                            uint32_t base, unsigned* sync, unsigned target) {
+    conv_tc_roles<ACT, POOL, RES, ROW, false>(&Y->tmx, &Y->tmw, &Y->tmy, &Y->tmr, *p, *sm, tmem_base, stage0, base, GridSync{sync, target});
+}
+
+__global__ void __launch_bounds__(kThreads, 1) conv_seq_kernel(const __grid_constant__ SeqParams sp) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[8], empty_bar[8], tfull_bar[2], tempty_bar[2];
+    __shared__ uint64_t sfull_bar[2], sfree_bar[2];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    // the current layer's parameters, copied out of the kernel's parameter block: the roles read them all the time, and a
+    // dynamically indexed parameter array is read through generic loads
+    __shared__ __align__(16) ConvTcParams p_s;
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* stage0 = smem_raw + (base - smem_u32(smem_raw));
+    const int warp = threadIdx.x >> 5;
+    const ConvBars sm{full_bar, empty_bar, tfull_bar, tempty_bar, sfull_bar, sfree_bar, &abort_s};
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        conv_tc_init_bars(sm, 8, false);
+    }
+    if (warp == kMmaWarp) {
+        tmem_alloc(&tmem_base_s, 512);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = tmem_base_s;
+
+#pragma unroll 1
+    for (int l = 0; l < sp.n_layers; l++) {
+        const SeqLayer& Y = sp.L[l];
+        if (l == 1 && threadIdx.x == 0) DLF_TRACE_POINT(sp.status, 20);
+        for (int i = threadIdx.x; i < static_cast<int>(sizeof(ConvTcParams) / 4); i += kThreads)
+            reinterpret_cast<int*>(&p_s)[i] = reinterpret_cast<const int*>(&Y.p)[i];
+        if (threadIdx.x == 0) {   // fresh barriers for this layer's ring (every role is past the previous layer: see the barrier below)
+            if (l > 0) conv_tc_init_bars(sm, 8, true);
+            tma_prefetch_desc(&Y.tmx);
+            tma_prefetch_desc(&Y.tmw);
+        }
+        __syncthreads();
+        if (l == 1 && threadIdx.x == 0) DLF_TRACE_POINT(sp.status, 21);
+        const unsigned target = static_cast<unsigned>(l) * gridDim.x;   // every CTA has finished the layers before this one
+#define DLF_SEQ_CASE(ACT, POOL, RES, ROW)                                                                      \
+    case ((ACT * 2 + POOL) * 2 + RES) * 2 + ROW:                                                               \
+        conv_seq_layer<ACT, POOL != 0, RES != 0, ROW != 0>(&Y, &p_s, &sm, tmem_base, stage0, base, sp.sync, target); \
+        break;
+        switch (Y.variant) {
+            DLF_SEQ_CASE(0, 0, 0, 0) DLF_SEQ_CASE(0, 0, 0, 1) DLF_SEQ_CASE(0, 0, 1, 0) DLF_SEQ_CASE(0, 0, 1, 1) DLF_SEQ_CASE(0, 1, 0, 0) DLF_SEQ_CASE(0, 1, 1, 0)
+            DLF_SEQ_CASE(1, 0, 0, 0) DLF_SEQ_CASE(1, 0, 0, 1) DLF_SEQ_CASE(1, 0, 1, 0) DLF_SEQ_CASE(1, 0, 1, 1) DLF_SEQ_CASE(1, 1, 0, 0) DLF_SEQ_CASE(1, 1, 1, 0)
+            DLF_SEQ_CASE(2, 0, 0, 0) DLF_SEQ_CASE(2, 0, 0, 1) DLF_SEQ_CASE(2, 0, 1, 0) DLF_SEQ_CASE(2, 0, 1, 1) DLF_SEQ_CASE(2, 1, 0, 0) DLF_SEQ_CASE(2, 1, 1, 0)
+            default: break;
+        }
+#undef DLF_SEQ_CASE
+        // the layer is finished on this CTA once its stores have completed and every role has left it
+        if (l == 0 && threadIdx.x == 0) DLF_TRACE_POINT(sp.status, 22);
+        if (l == 0 && threadIdx.x == 32 * kStoreWarp) DLF_TRACE_POINT(sp.status, 23);
+        if (warp == kStoreWarp) {
+            tma_store_wait_all();
+            asm volatile("fence.proxy.async;" ::: "memory");
+        }
+        if (l == 0 && threadIdx.x == 32 * kStoreWarp) DLF_TRACE_POINT(sp.status, 24);
+        __threadfence();
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+        if (l == 0 && threadIdx.x == 0) DLF_TRACE_POINT(sp.status, 25);
+        if (threadIdx.x == 0 && l + 1 < sp.n_layers) {
+            __threadfence();
+            atomicAdd(sp.sync, 1u);
+        }
+        if (l == 0 && threadIdx.x == 0) DLF_TRACE_POINT(sp.status, 26);
+    }
+    // the last CTA to leave puts the two counters back to zero for the next launch
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(sp.sync + 1, 1u) == gridDim.x - 1) {
+            sp.sync[0] = 0u;
+            sp.sync[1] = 0u;
+            __threadfence();
+        }
+    }
+    if (warp == kMmaWarp) {
+        if (abort_s) __nanosleep(20000);
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, 512);
     }
 }
 
@@ -609,12 +814,18 @@ bool conv_tc_supported(const ConvArgs& a) {
     return true;
 }
 
-int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStream_t s) {
+namespace {
+// Everything a launch of one layer needs: tensor maps, parameters, the kernel variant, shared memory, grid.
+struct ConvTcLaunch {
+    CUtensorMap tmx, tmw, tmy, tmr;
+    ConvTcParams p;
+    int act, pool, res, row, split;
+    size_t smem;
+    int grid;
+};
+
+int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcLaunch* out) {
     if (!conv_tc_supported(a_in)) return DLF_E_UNSUPPORTED;
-    {
-        int rc = conv_tc_init();
-        if (rc) return rc;
-    }
     // A 1x1 stride-1 convolution has no spatial structure: its N x H x W pixels are one list, cut into tiles of any
     // length, so that the persistent grid's rounds can be filled evenly (below) whatever the image size.
     ConvArgs a = a_in;
@@ -879,15 +1090,72 @@ int launch_conv_tc(const ConvArgs& a_in, int sm_count, int* status_dev, cudaStre
             if (rc) return rc;
         }
     }
-    const int grid = std::max(1, std::min(sm_count, p.n_work));
+    out->grid = std::max(1, std::min(sm_count, p.n_work));
     // never two of these CTAs on an SM: each may hold all of tensor memory
-    const size_t smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024 + (kABytes + 256 - p.a_bytes), 120 * 1024);
+    out->smem = std::max<size_t>(static_cast<size_t>(p.bias_off) + bias_bytes + 1024 + (kABytes + 256 - p.a_bytes), 120 * 1024);
 #ifdef DLF_TRACE
     fprintf(stderr, "conv_tc: tile %dx%dx%d rows %d BN %d x %d splits %d kgs %d kg %d kgroups %d stages %d out_bufs %d work %d grid %d\n", tl.tn, tl.th, tl.tw,
-            p.rows, p.BN, p.n_tiles_n, p.splits, p.kgs, p.kg, p.kgroups, p.stages, p.out_bufs, p.n_work, grid);
+            p.rows, p.BN, p.n_tiles_n, p.splits, p.kgs, p.kg, p.kgroups, p.stages, p.out_bufs, p.n_work, out->grid);
 #endif
-    const KernelFn fn = splits > 1 ? pick_split(a.act, p.tps == 3) : pick_kernel(a.act, a.pool != 0, a.res != nullptr, p.tps == 3);
-    cudaError_t e = launch_kernel(fn, grid, kThreads, smem, s, tmx, tmw, tmy, tmr, p);
+    out->tmx = tmx; out->tmw = tmw; out->tmy = tmy; out->tmr = tmr;
+    out->p = p;
+    out->act = a.act; out->pool = a.pool != 0; out->res = a.res != nullptr; out->row = p.tps == 3; out->split = splits > 1;
+    return DLF_OK;
+}
+}  // namespace
+
+int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s) {
+    int rc = conv_tc_init();
+    if (rc) return rc;
+    ConvTcLaunch L;
+    rc = conv_tc_prepare(a, sm_count, status_dev, &L);
+    if (rc) return rc;
+    const KernelFn fn = L.split ? pick_split(L.act, L.row != 0) : pick_kernel(L.act, L.pool != 0, L.res != 0, L.row != 0);
+    cudaError_t e = launch_kernel(fn, L.grid, kThreads, L.smem, s, L.tmx, L.tmw, L.tmy, L.tmr, L.p);
+    return e == cudaSuccess ? DLF_OK : cuda_fail(e);
+}
+
+int g_seq_cooperative = 0;
+bool conv_seq_layer_supported(const ConvArgs& a) { return conv_tc_supported(a); }
+int conv_seq_max_layers() { return kMaxSeq; }
+
+// Several dense convolutions as one persistent kernel on `sm_count` CTAs (a cooperative launch: every CTA must be resident,
+// they wait for one another between the layers).  `sync_dev`: two words of device memory that are zero between launches.
+int launch_conv_seq(const ConvArgs* layers, int n_layers, int sm_count, int* status_dev, unsigned* sync_dev, cudaStream_t s) {
+    if (n_layers < 1 || n_layers > kMaxSeq || !sync_dev) return DLF_E_PLAN;
+    int rc = conv_tc_init();
+    if (rc) return rc;
+    static SeqParams sp;   // (large: not on the stack; the launch copies it)
+    std::memset(&sp, 0, sizeof(sp));
+    size_t smem = 0;
+    for (int l = 0; l < n_layers; l++) {
+        ConvArgs a = layers[l];
+        a.splitk_ws = nullptr;   // no split reductions inside a multi-layer launch
+        a.splitk_bytes = 0;
+        ConvTcLaunch L;
+        rc = conv_tc_prepare(a, sm_count, status_dev, &L);
+        if (rc) return rc;
+        if (L.split || (L.pool && L.row)) return DLF_E_UNSUPPORTED;
+        SeqLayer& Y = sp.L[l];
+        Y.tmx = L.tmx; Y.tmw = L.tmw; Y.tmy = L.tmy; Y.tmr = L.tmr;
+        Y.p = L.p;
+        Y.variant = ((L.act * 2 + L.pool) * 2 + L.res) * 2 + L.row;
+        smem = std::max(smem, L.smem);
+    }
+    sp.n_layers = n_layers;
+    sp.sync = sync_dev;
+    sp.status = status_dev;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(sm_count));
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = g_seq_cooperative ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, conv_seq_kernel, sp);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 
@@ -909,6 +1177,10 @@ int conv_tc_init() {
                 cudaError_t e = cudaFuncSetAttribute(pick_split(act, row != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
                 if (e != cudaSuccess) return cuda_fail(e);
             }
+        {
+            cudaError_t e = cudaFuncSetAttribute(conv_seq_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+            if (e != cudaSuccess) return cuda_fail(e);
+        }
         attr_set[dev] = true;
     }
     return DLF_OK;

@@ -108,6 +108,10 @@ int launch_fc(const void* x, const void* w, const float* bias, void* y, int N, i
 bool conv_tc_supported(const ConvArgs& a);
 bool chain_tc_layer_supported(int cin, int cout, int k);
 int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_t s);
+// Several layers as one persistent kernel with device-wide barriers between them (conv_tc.cu).
+bool conv_seq_layer_supported(const ConvArgs& a);
+int conv_seq_max_layers();
+int launch_conv_seq(const ConvArgs* layers, int n_layers, int sm_count, int* status_dev, unsigned* sync_dev, cudaStream_t s);
 
 // stem_tc.cu
 bool stem_tc_supported(const ConvArgs& a);

@@ -296,3 +296,42 @@ def test_two_fused_blocks_in_a_row_and_partial_groups_are_refused():
         with pytest.raises(B.DlfError) as e:
             B.net_set_plan(sess.net, ends, [sms()] * len(ends))
         assert e.value.status == B.E_PLAN
+
+
+# ---- groups handed over through L2: one persistent kernel, a device-wide barrier between the layers -------------------
+def _bottleneck_with_projection():
+    """A down-sampling bottleneck (stride on the 3x3, 1x1/2 projection of the block input added before the ReLU),
+    a second block whose skip is the first block's output, then a pooled 3x3 layer."""
+    return [_conv(32, 16, 1, src=-1), _conv(16, 16, 3, stride=2, src=0), _conv(32, 64, 1, stride=2, pad=0, act="none", src=-1),
+            _conv(16, 64, 1, src=1, res_src=2), _conv(64, 16, 1, src=3), _conv(16, 16, 3, src=4),
+            _conv(16, 64, 1, src=5, res_src=3), _conv(64, 72, 3, src=6, pool=2)]
+
+
+def test_l2_groups_every_contiguous_plan():
+    layers = _bottleneck_with_projection()
+    n = len(layers)
+    sess, xd, ref = _mk(layers, "l2group", 3, 18, 22, 32)
+    B.net_set_option(sess.net, B.OPT_GROUP_KERNEL, 2)
+    G.check_plan(sess, xd, ref, list(range(n)), [sms()] * n, "unfused")
+    ran = 0
+    for mask in range(1 << (n - 1)):
+        if mask % 5 not in (0, 3) and mask != (1 << (n - 1)) - 1:   # a sample of the 128 plans, plus all-in-one
+            continue
+        ends = [i for i in range(n - 1) if mask >> i & 1] + [n - 1]
+        for s in (sms(), 5):
+            G.check_plan(sess, xd, ref, ends, [s] * len(ends), "L2 groups %s S=%d" % (ends, s))
+            ran += 1
+    assert ran > 20
+    sess.set_plan([n - 1], [sms()])
+    assert sess.kernels() == ["conv_seq"]
+    for _ in range(3):   # the barrier counters are back at zero after every launch
+        G.check_plan(sess, xd, ref, [2, n - 1], [7, sms()], "L2 groups, repeated")
+
+
+def test_group_kernel_option_chooses_the_hand_over():
+    layers = [_conv(128, 128, 1, src=-1), _conv(128, 128, 3, src=0), _conv(128, 128, 1, src=1, res_src=-1)]
+    sess, xd, ref = _mk(layers, "handover", 2, 14, 14, 128)
+    for opt, kernel in ((0, "conv_seq"), (1, "chain_tc"), (2, "conv_seq")):
+        B.net_set_option(sess.net, B.OPT_GROUP_KERNEL, opt)
+        G.check_plan(sess, xd, ref, [2], [sms()], "option %d" % opt)
+        assert sess.kernels() == [kernel]
