@@ -151,6 +151,14 @@ int dlf_net_bruteforce(dlf_net* net, const dlf_search_params* params, const void
                        void* stream, int* n_groups, int32_t* group_end, int32_t* sm_count,
                        float* best_ms);
 
+/* The search's dynamic programme alone, on a table the caller supplies (host only; no net, no device): ms is
+ * [n_layers][max_group_len][n_sm_choices], the time of span a..a+len-1 on sm_choices[c] SMs at
+ * ms[(a * max_group_len + len - 1) * n_sm_choices + c], negative for a group that cannot run.  Returns the contiguous
+ * partition with the least total time (Sec. V: a plan's time is the sum of its blocks' times), each group with the SM
+ * count that gave its best time.  DLF_E_PLAN if no partition is possible. */
+int dlf_bruteforce_table(int n_layers, int max_group_len, int n_sm_choices, const int32_t* sm_choices, const float* ms,
+                         int* n_groups, int32_t* group_end, int32_t* sm_count, float* best_ms);
+
 /* Times layers first..last as ONE candidate group on sm_count SMs, outside any plan (the single-layer
  * micro-benchmark of the paper's characterisation, Sec. II-B, and one cell of the reduced brute-force
  * search, Sec. V): median device time of one launch, taken over `iters` timings of four back-to-back
@@ -171,6 +179,12 @@ int dlf_net_run_host(dlf_net* net, const void* in_f16_host, void* out_f16_host, 
 /* Waits for the stream and reports a device-side bounded wait that gave up (DLF_E_TIMEOUT)
  * or a CUDA error from the kernels enqueued so far. */
 int dlf_net_sync(dlf_net* net, void* stream);
+
+/* Self-test of the bounded device-side waits: enqueues a one-CTA kernel that waits - through the very routine every kernel's
+ * waits use - at a barrier nothing arrives at, with the limit lowered from one second to limit_us microseconds.  The wait
+ * gives up, records its code in the net's status word and the kernel ends normally; the next dlf_net_sync on that stream
+ * returns DLF_E_TIMEOUT (and clears the word), later runs are unaffected.  Nothing traps, nothing spins beyond the limit. */
+int dlf_net_debug_stall(dlf_net* net, int limit_us, void* stream);
 
 /* Times `iters` runs with CUDA events on `stream` after `warmup` untimed ones.  If flush_dev is
  * non-NULL its flush_bytes are overwritten before every run, outside the timed interval, to

@@ -67,10 +67,12 @@ def lib():
             "dlf_net_tuner_may_fuse": (C.c_int, [vp, C.c_int, C.c_int, C.c_int, C.c_int]),
             "dlf_net_autotune": (C.c_int, [vp, C.POINTER(TunerParams), ip, i32p, i32p]),
             "dlf_net_bruteforce": (C.c_int, [vp, C.POINTER(SearchParams), vp, vp, ip, i32p, i32p, fp]),
+            "dlf_bruteforce_table": (C.c_int, [C.c_int, C.c_int, C.c_int, i32p, fp, ip, i32p, i32p, fp]),
             "dlf_net_time_span": (C.c_int, [vp, C.c_int, C.c_int, C.c_int, vp, vp, C.c_int, C.c_int, C.c_int, fp]),
             "dlf_net_run": (C.c_int, [vp, vp, vp, vp]),
             "dlf_net_run_host": (C.c_int, [vp, vp, vp, vp]),
             "dlf_net_sync": (C.c_int, [vp, vp]),
+            "dlf_net_debug_stall": (C.c_int, [vp, C.c_int, vp]),
             "dlf_net_time": (C.c_int, [vp, vp, vp, vp, C.c_int, C.c_int, vp, C.c_size_t, fp, fp, fp]),
             "dlf_net_boundary_tensor": (C.c_int, [vp, C.c_int, C.POINTER(vp), i64p]),
             "dlf_net_group_model": (C.c_int, [vp, C.c_int, i64p, i64p, C.POINTER(C.c_double), ip]),
@@ -199,6 +201,16 @@ def net_bruteforce(net, n_layers, sm_choices, max_group_len, in_ptr, stream=None
     return list(e[:n.value]), list(s[:n.value]), ms.value
 
 
+def bruteforce_table(n_layers, max_group_len, sm_choices, ms):
+    """ms[a][len - 1][c]: time of span a..a+len-1 on sm_choices[c] SMs, negative = cannot run."""
+    flat = [float(ms[a][l][c]) for a in range(n_layers) for l in range(max_group_len) for c in range(len(sm_choices))]
+    n, best = C.c_int(), C.c_float()
+    e, s = (C.c_int32 * n_layers)(), (C.c_int32 * n_layers)()
+    _check(lib().dlf_bruteforce_table(n_layers, max_group_len, len(sm_choices), _i32(sm_choices), (C.c_float * len(flat))(*flat),
+                                      C.byref(n), e, s, C.byref(best)), "dlf_bruteforce_table")
+    return list(e[:n.value]), list(s[:n.value]), best.value
+
+
 def net_time_span(net, first, last, sm_count, in_ptr, stream=None, warmup=2, iters=5, prepare=True):
     ms = C.c_float()
     _check(lib().dlf_net_time_span(net, first, last, sm_count, in_ptr, stream, warmup, iters, 1 if prepare else 0,
@@ -216,6 +228,10 @@ def net_run_host(net, in_host_ptr, out_host_ptr, stream=None):
 
 def net_sync(net, stream=None):
     _check(lib().dlf_net_sync(net, stream), "dlf_net_sync")
+
+
+def net_debug_stall(net, limit_us, stream=None):
+    _check(lib().dlf_net_debug_stall(net, limit_us, stream), "dlf_net_debug_stall")
 
 
 def net_time(net, in_ptr, out_ptr, n_groups, stream=None, warmup=3, iters=10, flush_ptr=None, flush_bytes=0,

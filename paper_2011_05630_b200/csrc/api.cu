@@ -597,6 +597,37 @@ static int layer_sms(const Layer& l, const dlf_tuner_params& p, int s_max) {
 
 }  // namespace dlf
 
+namespace dlf {
+// The search's second half: given the best time t[a][len-1] of every span a..a+len-1 (infinity: cannot run) and the SM
+// count that reached it, the contiguous partition with the least total time (a plan's time is the sum of its groups').
+static int solve_partition(int n, int max_len, const std::vector<std::vector<float>>& t, const std::vector<std::vector<int>>& ts, int* n_groups,
+                           int32_t* group_end, int32_t* sm_count, float* best_ms) {
+    const float inf = std::numeric_limits<float>::infinity();
+    std::vector<float> best(n + 1, inf);
+    std::vector<int> from(n + 1, -1);
+    best[0] = 0.0f;
+    for (int i = 1; i <= n; i++)
+        for (int len = 1; len <= max_len && len <= i; len++) {
+            const int a = i - len;
+            if (best[a] == inf || t[a][len - 1] == inf) continue;
+            if (best[a] + t[a][len - 1] < best[i]) { best[i] = best[a] + t[a][len - 1]; from[i] = a; }
+        }
+    if (best[n] == inf) return DLF_E_PLAN;
+    std::vector<int> cuts;
+    for (int i = n; i > 0; i = from[i]) cuts.push_back(i);
+    std::reverse(cuts.begin(), cuts.end());
+    int a = 0;
+    for (size_t g = 0; g < cuts.size(); g++) {
+        group_end[g] = cuts[g] - 1;
+        sm_count[g] = ts[a][cuts[g] - a - 1];
+        a = cuts[g];
+    }
+    *n_groups = static_cast<int>(cuts.size());
+    if (best_ms) *best_ms = best[n];
+    return DLF_OK;
+}
+}  // namespace dlf
+
 dlf_net::~dlf_net() {
     graph.drop();
     graph_timed.drop();
@@ -913,6 +944,13 @@ int dlf_net_sync(dlf_net* net, void* stream) {
     return DLF_OK;
 }
 
+int dlf_net_debug_stall(dlf_net* net, int limit_us, void* stream) {
+    if (!net || limit_us < 1 || limit_us > 1000000) return DLF_E_INVALID_ARG;
+    if (!net->ws) return DLF_E_WORKSPACE;
+    return launch_stall(reinterpret_cast<int*>(net->ws + net->status_off), static_cast<unsigned long long>(limit_us) * 1000ull,
+                        static_cast<cudaStream_t>(stream));
+}
+
 int dlf_net_run_host(dlf_net* net, const void* in_f16_host, void* out_f16_host, void* stream) {
     if (!net || !in_f16_host || !out_f16_host) return DLF_E_INVALID_ARG;
     int rc = check_ready(net);
@@ -1092,29 +1130,25 @@ int dlf_net_bruteforce(dlf_net* net, const dlf_search_params* sp, const void* in
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     if (rc) return rc;
-    // dynamic programme over contiguous partitions
-    std::vector<float> best(n + 1, inf);
-    std::vector<int> from(n + 1, -1);
-    best[0] = 0.0f;
-    for (int i = 1; i <= n; i++)
-        for (int len = 1; len <= sp->max_group_len && len <= i; len++) {
-            const int a = i - len;
-            if (best[a] == inf || t[a][len - 1] == inf) continue;
-            if (best[a] + t[a][len - 1] < best[i]) { best[i] = best[a] + t[a][len - 1]; from[i] = a; }
-        }
-    if (best[n] == inf) return DLF_E_PLAN;
-    std::vector<int> cuts;
-    for (int i = n; i > 0; i = from[i]) cuts.push_back(i);
-    std::reverse(cuts.begin(), cuts.end());
-    int a = 0;
-    for (size_t g = 0; g < cuts.size(); g++) {
-        group_end[g] = cuts[g] - 1;
-        sm_count[g] = ts[a][cuts[g] - a - 1];
-        a = cuts[g];
-    }
-    *n_groups = static_cast<int>(cuts.size());
-    if (best_ms) *best_ms = best[n];
+    rc = solve_partition(n, sp->max_group_len, t, ts, n_groups, group_end, sm_count, best_ms);
+    if (rc) return rc;
     return dlf_net_sync(net, s);
+}
+
+int dlf_bruteforce_table(int n_layers, int max_group_len, int n_sm_choices, const int32_t* sm_choices, const float* ms, int* n_groups,
+                         int32_t* group_end, int32_t* sm_count, float* best_ms) {
+    if (n_layers < 1 || max_group_len < 1 || n_sm_choices < 1 || !sm_choices || !ms || !n_groups || !group_end || !sm_count) return DLF_E_INVALID_ARG;
+    const float inf = std::numeric_limits<float>::infinity();
+    std::vector<std::vector<float>> t(n_layers, std::vector<float>(max_group_len, inf));
+    std::vector<std::vector<int>> ts(n_layers, std::vector<int>(max_group_len, 0));
+    for (int a = 0; a < n_layers; a++)
+        for (int len = 1; len <= max_group_len && a + len <= n_layers; len++)
+            for (int c = 0; c < n_sm_choices; c++) {
+                const float m = ms[(static_cast<size_t>(a) * max_group_len + (len - 1)) * n_sm_choices + c];
+                if (m >= 0.0f && m < t[a][len - 1]) { t[a][len - 1] = m; ts[a][len - 1] = sm_choices[c]; }
+            }
+    return solve_partition(n_layers, max_group_len, t, ts, n_groups, group_end, sm_count, best_ms);
+
 }
 
 int dlf_net_boundary_tensor(const dlf_net* net, int layer, const void** dev_ptr, int64_t shape[4]) {

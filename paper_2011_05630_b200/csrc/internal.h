@@ -104,6 +104,8 @@ int launch_gavgpool(const void* x, void* y, int N, int H, int W, int C, int sm_c
 int launch_fc(const void* x, const void* w, const float* bias, void* y, int N, int K, int M, int act, int sm_count,
               cudaStream_t s);
 
+int launch_stall(int* status_dev, unsigned long long limit_ns, cudaStream_t s);
+
 // conv_tc.cu
 bool conv_tc_supported(const ConvArgs& a);
 bool chain_tc_layer_supported(int cin, int cout, int k);

@@ -422,4 +422,24 @@ int launch_fc(const void* x, const void* w, const float* bias, void* y, int N, i
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 
+// Self-test of the bounded waits: one CTA waits, with the waits' own routine, at a barrier that nothing ever arrives at.
+// The wait has to give up after `limit_ns`, record its code in the status word and let the kernel end normally.
+__global__ void stall_kernel(int* status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_s;
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        mbar_init(&bar, 1);
+        fence_barrier_init();
+    }
+    __syncthreads();
+    mbar_wait(&bar, 0u, &abort_s, status, 0xd00, limit_ns);
+}
+
+int launch_stall(int* status_dev, unsigned long long limit_ns, cudaStream_t s) {
+    stall_kernel<<<1, 64, 0, s>>>(status_dev, limit_ns);
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? DLF_OK : cuda_fail(e);
+}
+
 }  // namespace dlf

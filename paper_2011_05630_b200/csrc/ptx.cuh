@@ -83,7 +83,7 @@ constexpr uint64_t kWaitLimitNs = 1000000000ull;  // one second
 // start to sleep.  (try_wait with a suspend-time hint instead of this loop was measured 1-3 % slower.)
 template <bool HOT = false>
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int code) {
+                                          int* status, int code, uint64_t limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     uint64_t t0 = 0;   // the global timer is read only once a wait has lasted a while
     uint32_t spins = 0;
@@ -95,7 +95,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             if (*abort_flag) return false;
             const uint64_t now = global_ns();
             if (t0 == 0) t0 = now;
-            if (now - t0 > kWaitLimitNs) {
+            if (now - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicCAS(status, 0, code);
                 return false;

@@ -139,3 +139,41 @@ def test_autotune_equals_restated_algorithm1(name, layers, batch, crit):
     if name == "two_layer" and crit == 1e30:      # the two narrow 3x3 layers: the fused kernel is estimated to pay
         assert got[0] == [1]
     B.net_destroy(net)
+
+
+# ---- the search's dynamic programme against exhaustive enumeration --------------------------------------------------
+def test_bruteforce_table_on_the_hand_worked_example():
+    # the table of tests/test_oracle_model.py: three layers, core counts {1, 2}
+    table = {(0, 0, 1): 5, (0, 0, 2): 3, (1, 1, 1): 4, (1, 1, 2): 2.5, (2, 2, 1): 6, (2, 2, 2): 3.5,
+             (0, 1, 1): 6, (0, 1, 2): 4, (1, 2, 1): 7, (1, 2, 2): 5.5}
+    ms = [[[table.get((a, a + l, m), -1.0) for m in (1, 2)] for l in range(3)] for a in range(3)]
+    assert B.bruteforce_table(3, 3, [1, 2], ms) == ([1, 2], [2, 2], 7.5)     # [0,1][2] -> 4 + 3.5
+    assert B.bruteforce_table(3, 1, [1, 2], [[r[0]] for r in ms]) == ([0, 1, 2], [2, 2, 2], 9.0)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_bruteforce_table_equals_exhaustive_search(seed):
+    import random
+    rnd = random.Random(seed)
+    n, q, max_len = rnd.randint(1, 6), rnd.randint(1, 3), rnd.randint(1, 4)
+    choices = sorted(rnd.sample(range(1, 149), q))
+    ms = [[[(-1.0 if (l > 0 and rnd.random() < 0.3) or a + l >= n else round(rnd.uniform(0.5, 9.0), 3)) for _ in choices]
+           for l in range(max_len)] for a in range(n)]
+
+    def group_time(a, e, m):
+        if e - a >= max_len:
+            return None
+        v = ms[a][e - a][choices.index(m)]
+        return None if v < 0 else v
+
+    want = model.best_plan_exhaustive(n, choices, group_time, max_len=max_len)
+    ends, smc, best = B.bruteforce_table(n, max_len, choices, ms)
+    assert best == pytest.approx(want[0], rel=1e-5)
+    total = sum(group_time(a, e, m) for a, e, m in zip([0] + [x + 1 for x in ends[:-1]], ends, smc))   # the plan returned costs what is claimed
+    assert total == pytest.approx(best, rel=1e-5)
+
+
+def test_bruteforce_table_without_a_partition():
+    import ctypes as C
+    assert B.lib().dlf_bruteforce_table(2, 2, 1, (C.c_int32 * 1)(4), (C.c_float * 4)(1.0, -1.0, -1.0, -1.0), C.byref(C.c_int()),
+                                        (C.c_int32 * 2)(), (C.c_int32 * 2)(), None) == B.E_PLAN

@@ -13,6 +13,7 @@ import pytest
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
+from oracle import executor as orc
 from paper_2011_05630_b200 import binding as B, synth
 from paper_2011_05630_b200.runtime import Session
 from tests import gpu_util as G
@@ -37,10 +38,12 @@ def test_static_scratch_entry_matches_workspace_entry_twice():
         x = synth.network_input(tag, n, h, w, 32)
         xd = sess.upload(x)
         want = sess.run(xd).cpu().numpy()
+        G.compare(want, orc.run_network(layers, params, x)[-1], "workspace entry against the CPU checker, call %d" % call)
         y.fill_(float("nan"))
         B.conv_chain_run_static(layers, n, h, w, xd.data_ptr(), w_ptrs, b_ptrs, y.data_ptr(), sms,
                                 torch.cuda.current_stream().cuda_stream)
         G.compare(y.cpu().numpy(), want, "static scratch, call %d" % call)
+        G.compare(y.cpu().numpy(), orc.run_network(layers, params, x)[-1], "static scratch against the CPU checker, call %d" % call)
     sess.close()
 
 
