@@ -45,6 +45,55 @@ def vgg16(classes=1000):
     return _finish(L)
 
 
+def vgg19(classes=1000):
+    """VGG-19 (the paper's Table 2 workload): 16 conv3x3 + bias + ReLU in five stages (2, 2, 4, 4, 4), 2x2 max-pool
+    fused after each stage, then the same three fully connected layers as VGG-16."""
+    L, cin = [], 3
+    for width, reps in ((64, 2), (128, 2), (256, 4), (512, 4), (512, 4)):
+        for r in range(reps):
+            L.append(_layer("conv", cin, width, 3, act="relu", pool=2 if r == reps - 1 else 0))
+            cin = width
+    L.append(_layer("fc", 7 * 7 * 512, 4096, act="relu"))
+    L.append(_layer("fc", 4096, 4096, act="relu"))
+    L.append(_layer("fc", 4096, classes))
+    return _finish(L)
+
+
+def resnet18(classes=1000):
+    """ResNet-18 (Table 2): 7x7/2 stem + 3x3/2 max-pool, basic blocks [2,2,2,2] of two 3x3 convolutions (stride on the
+    first; list order per block: first 3x3, 1x1/2 projection if any, second 3x3 + add + ReLU), global average pool, FC:
+    20 convolutions."""
+    L = [_layer("conv", 3, 64, 7, stride=2, pad=3, act="relu"),
+         _layer("maxpool", 64, 64, 3, stride=2, pad=1)]
+    cin, block_in = 64, 1
+    for stage, width in enumerate((64, 128, 256, 512)):
+        for b in range(2):
+            s = 2 if (b == 0 and stage > 0) else 1
+            L.append(_layer("conv", cin, width, 3, stride=s, act="relu", src=block_in))
+            first = len(L) - 1
+            skip = block_in
+            if s == 2:
+                L.append(_layer("conv", cin, width, 1, stride=s, pad=0, src=block_in))
+                skip = len(L) - 1
+            L.append(_layer("conv", width, width, 3, act="relu", src=first, res_src=skip))
+            block_in, cin = len(L) - 1, width
+    L.append(_layer("gavgpool", cin, cin))
+    L.append(_layer("fc", cin, classes))
+    return _finish(L)
+
+
+def alexnet(classes=1000):
+    """AlexNet in its single-tower form (the variant whose operation count matches Table 2): 11x11/4 pad 2 -> 64,
+    3x3/2 max-pool, 5x5 pad 2 -> 192, 3x3/2 max-pool, three 3x3 (384, 256, 256), 3x3/2 max-pool, FC 9216-4096-4096-classes;
+    bias + ReLU after every convolution and hidden FC."""
+    L = [_layer("conv", 3, 64, 11, stride=4, pad=2, act="relu"), _layer("maxpool", 64, 64, 3, stride=2, pad=0),
+         _layer("conv", 64, 192, 5, pad=2, act="relu"), _layer("maxpool", 192, 192, 3, stride=2, pad=0),
+         _layer("conv", 192, 384, 3, act="relu"), _layer("conv", 384, 256, 3, act="relu"), _layer("conv", 256, 256, 3, act="relu"),
+         _layer("maxpool", 256, 256, 3, stride=2, pad=0),
+         _layer("fc", 6 * 6 * 256, 4096, act="relu"), _layer("fc", 4096, 4096, act="relu"), _layer("fc", 4096, classes)]
+    return _finish(L)
+
+
 def resnet50(classes=1000):
     """7x7/2 stem + 3x3/2 max-pool, bottlenecks [3,4,6,3] (stride on the 3x3; list
     order per block: reduce, 3x3, projection if any, expand + add + ReLU), global

@@ -1,4 +1,5 @@
-"""GPU parity at the full workload sizes: VGG-16 b8, ResNet-50 b1/b32, MobileNetV2 b1/b64.
+"""GPU parity at the full workload sizes: VGG-16 b8, ResNet-50 b1/b32, MobileNetV2 b1/b64, and the paper's other Table 2
+networks (VGG-19, ResNet-18, AlexNet).
 
 The device runs the whole batch in the launch configuration the benchmark times; the CPU
 checker, whose images are independent (pinned bit-exactly on the CPU), runs a sample of the
@@ -16,7 +17,8 @@ from paper_2011_05630_b200.runtime import Session
 from tests import gpu_util as G
 
 NETS = [("vgg16", nw.vgg16, 8), ("resnet50", nw.resnet50, 1), ("resnet50", nw.resnet50, 32),
-        ("mobilenet_v2", nw.mobilenet_v2, 1), ("mobilenet_v2", nw.mobilenet_v2, 64)]
+        ("mobilenet_v2", nw.mobilenet_v2, 1), ("mobilenet_v2", nw.mobilenet_v2, 64),
+        ("vgg19", nw.vgg19, 8), ("resnet18", nw.resnet18, 32), ("alexnet", nw.alexnet, 32)]
 
 
 @pytest.mark.parametrize("name,builder,batch", NETS, ids=["%s_b%d" % (n, b) for n, _, b in NETS])
@@ -34,6 +36,14 @@ def test_network_every_boundary(name, builder, batch):
     todo = [("unfused", None, None)]
     ends, smc = plans.tuned_plan(sess.net, len(layers))
     todo.append(("tuned", ends, smc))
+    if name in ("resnet50", "resnet18"):   # one group per residual block (its layers handed over through L2), stem and tail apart
+        ends = [0, 1]
+        for i in range(2, len(layers) - 2):
+            if layers[i]["res_src"] != -2:
+                ends.append(i)
+        ends += [len(layers) - 2, len(layers) - 1]
+        assert len(ends) == (16 if name == "resnet50" else 8) + 4
+        todo.append(("block-fused", ends, [sms] * len(ends)))
     if name == "mobilenet_v2":   # every inverted-residual block as one group, the wide ones the tuner leaves apart too
         ends, i = [], 0
         while i < len(layers):

@@ -76,6 +76,18 @@ def test_table2_operation_counts(golden_dir, name, layers, key):
     assert abs(total / len(convs) - float(p["table2.%s.avg" % key])) <= 0.0051, total / len(convs)
 
 
+def test_workload_recipes_are_the_table2_networks():
+    """The library's own builders (run on the GPU and timed) have the convolution layers of the builders above."""
+    key = lambda l: (l["op"], l["cin"], l["cout"], l["kh"], l["stride"], l["pad"])
+    for mine, theirs in ((vgg19(), nw.vgg19()), (resnet18(), nw.resnet18()), (alexnet_single_tower(), nw.alexnet())):
+        convs = lambda layers: [key(l) for l in layers if l["op"] == "conv"]
+        assert convs(mine) == convs(theirs)
+    assert [l["src"] for l in resnet18()] == [l["src"] for l in nw.resnet18()[:len(resnet18())]]   # the skip wiring too
+    for layers, hw in ((nw.vgg19(), 224), (nw.resnet18(), 224), (nw.alexnet(), 224)):
+        shapes = model.infer_shapes(layers, 1, hw, hw, 3)
+        assert shapes[-1] == (1, 1, 1, 1000)
+
+
 def test_equal_op_count_triple_of_sec4a():
     a = model.eq1_conv_ops(224, 224, 3, 3, 32, 32)
     assert a == model.eq1_conv_ops(112, 112, 3, 3, 64, 64) == model.eq1_conv_ops(56, 56, 3, 3, 128, 128)
