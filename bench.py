@@ -252,6 +252,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--groups", action="store_true", help="print the per-group table to stderr")
     ap.add_argument("--ablation", action="store_true", help="also time the strategies of the paper's ablation (Table 3); table to stderr")
+    ap.add_argument("--sm-sweep", action="store_true", help="also time the no-fusion plan at one network-wide SM count per run (the paper's Fig. 'Motivation' (a)); table to stderr")
     ap.add_argument("--layers", action="store_true", help="print a per-layer table (each layer alone, precise times) to stderr")
     ap.add_argument("--op-critical", type=float, default=None, help="override Algorithm 1's critical operation count per SM")
     args = ap.parse_args()
@@ -341,6 +342,22 @@ def main():
                 sys.stderr.write("| %s | %d | %d | %.4f | %.0f | %.2f |\n" % (r["strategy"], r["n_groups"], r["sm_count"], r["ms_per_step"],
                                                                             r["value"], r["speedup_over_strategy_1"]))
 
+    sm_sweep = None
+    if args.sm_sweep:   # one SM count for the whole network, no fusion: how many cores the network as a whole wants
+        sm_sweep = []
+        k_steps = max(3, min(args.steps, 20))
+        for f in plans.sm_fractions(sms):
+            sess.set_plan(list(range(len(layers))), [f] * len(layers))
+            barrier()
+            ms = time_plan(sess, B, torch, xd, k_steps, 3, flush, stream)
+            barrier()
+            value, total_ms = D.job_throughput(sum(ms), batch * k_steps, device=sess.device)
+            sm_sweep.append({"sm_count": f, "ms_per_step": total_ms / k_steps, "value": value})
+        if rank == 0:
+            sys.stderr.write("---- network-wide SM count, no fusion ----\n| S | ms / step | images/s |\n|---|---|---|\n")
+            for r in sm_sweep:
+                sys.stderr.write("| %d | %.4f | %.0f |\n" % (r["sm_count"], r["ms_per_step"], r["value"]))
+
     # end to end through the host-buffer entry point: pinned host input, H2D, run, D2H, per step
     sess.set_plan(t_ends, t_sms)
     xh = torch.from_numpy(x.view(np.int16)).pin_memory()
@@ -417,6 +434,8 @@ def main():
                 "paper_context": "3.6x-7.9x over no-fusion/MP=1 on a Cambricon MLU100 (other hardware)"}
         if ablation is not None:
             line["ablation"] = ablation
+        if sm_sweep is not None:
+            line["sm_sweep"] = sm_sweep
         if "bruteforce" in results:
             line["bruteforce"] = results["bruteforce"]
             line["tuned_over_bruteforce"] = tuned["value"] / results["bruteforce"]["value"]

@@ -9,8 +9,10 @@ takes for every layer the smallest SM count whose time is within `slack` of the 
     S = kappa_c * log2(C_out) + kappa_o * log2(ops) + kappa0          (least squares)
 
 which is Eq. 5's proportionality with its two weights and the affine map to an SM count fitted together
-(alpha = kappa_c / kappa, beta = kappa_o / kappa for any common scale kappa).  Only argument marshalling and the
-fit happen here; every timed step runs inside libdlfusion.so.
+(alpha = kappa_c / kappa, beta = kappa_o / kappa for any common scale kappa).  It also times the smaller layers on ONE
+SM and reads off Algorithm 1's OpCount_critical as the paper defines it (Sec. IV-C): the operation count from which a
+single core's throughput stays within a given fraction of its best.  Only argument marshalling and the fits happen here;
+every timed step runs inside libdlfusion.so.
 
     python -m paper_2011_05630_b200.characterise [--quick]
 """
@@ -68,6 +70,20 @@ def fit(rows, slack=0.05):
     return float(coef[0]), float(coef[1]), float(coef[2]), rms
 
 
+def critical_ops(single, frac=0.8):
+    """single: (ops, seconds on one SM) per layer.  The smallest operation count from which every layer reaches `frac` of
+    the best single-SM throughput seen (Sec. IV-C: where single-core efficiency saturates)."""
+    rows = sorted(single)
+    thr = [o / t for o, t in rows]
+    best = max(thr)
+    crit = rows[-1][0]
+    for (o, _), r in zip(reversed(rows), reversed(thr)):
+        if r < frac * best:
+            break
+        crit = o
+    return float(crit), float(best)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--quick", action="store_true", help="a third of the sweep")
@@ -75,17 +91,24 @@ def main():
     args = ap.parse_args()
     from . import binding as B, plans
     choices = plans.sm_fractions(B.device_sm_count())
-    rows = []
+    rows, single = [], []
     for n, hw, c, k in sweep_layers(args.quick):
         ops, times = time_layer(n, hw, c, k, choices)
         rows.append((c, ops, choices, times))
         best = min(times)
-        print("n %2d  %3dx%-3d c %3d k%d  ops %.3g  best %.1f us at S=%d" % (
-            n, hw, hw, c, k, ops, best * 1e3, choices[times.index(best)]), flush=True)
+        one = None
+        if ops <= 2e10:   # one SM: up to ~150 times longer than on the whole chip
+            one = time_layer(n, hw, c, k, [1])[1][0]
+            single.append((ops, one * 1e-3))
+        print("n %2d  %3dx%-3d c %3d k%d  ops %.3g  best %.1f us at S=%d%s" % (
+            n, hw, hw, c, k, ops, best * 1e3, choices[times.index(best)],
+            "" if one is None else "  one SM %.1f us (%.2f TFLOP/s)" % (one * 1e3, ops / (one * 1e-3) / 1e12)), flush=True)
     kc, ko, k0, rms = fit(rows, args.slack)
+    crit, best_thr = critical_ops(single)
     print(json.dumps({"layers": len(rows), "sm_choices": choices, "kappa_c": kc, "kappa_o": ko, "kappa0": k0,
                       "alpha_over_beta": kc / ko if ko else None, "rms_error_sms": rms,
-                      "paper_alpha_over_beta": 0.316 / 0.659}))
+                      "paper_alpha_over_beta": 0.316 / 0.659, "op_critical_per_sm": crit,
+                      "best_single_sm_tflops": best_thr / 1e12, "paper_op_critical": "10^1.25 G operations per core (MLU100)"}))
 
 
 if __name__ == "__main__":

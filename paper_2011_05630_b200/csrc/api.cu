@@ -409,11 +409,13 @@ static bool make_group(const dlf_net* net, int first, int last, int sms, Group* 
 // ---- what the tuner may propose as one group --------------------------------------------------------------------
 // Algorithm 1 grows a block while the layers can run as one kernel AND that kernel is expected to pay (Sec. IV-B: fusing
 // helps layers with few operations and hurts heavy ones).  For a dense chain the estimate is the fused kernel's own cost
-// model (the tiler's SM clocks at 1.9 GHz) against one kernel per layer: the slower of a layer's operations at 600 TFLOP/s
-// and its bytes at 5.5 TB/s (what the single-layer kernel reaches on this chip) plus 5.5 us per kernel boundary.
-// Inverted-residual blocks follow the measured rule on the hidden width.  Groups handed over through L2 are proposed only
-// when the option asks for them (measured: a device-wide barrier per layer is no cheaper than a kernel boundary).
-// `prefix`: the layers may also be the beginning of a pattern that can still grow into a group.
+// model (the tiler's SM clocks at 1.9 GHz, plus one kernel boundary) against one kernel per layer: the slower of a layer's
+// operations at 600 TFLOP/s and its bytes at 5.5 TB/s (what the single-layer kernel reaches on this chip) plus 7 us of
+// fixed cost per kernel (measured: no single-layer kernel takes less inside a network); the group must win by a tenth.
+// A chain may not swallow the expansion layer of an inverted-residual block (the layer a depthwise convolution reads):
+// that block fuses better as a whole.  Inverted-residual blocks follow the measured rule on the hidden width.  Groups
+// handed over through L2 are proposed only when the option asks for them (measured: a device-wide barrier per layer is no
+// cheaper than a kernel boundary).  `prefix`: the layers may also be the beginning of a pattern that can still grow.
 static bool tuner_may_fuse(const dlf_net* net, int first, int last, bool prefix, int s_max) {
     if (first == last) return true;
     if (net->opt_no_tc) return false;
@@ -421,6 +423,9 @@ static bool tuner_may_fuse(const dlf_net* net, int first, int last, bool prefix,
     if (net->opt_group_kernel == 2 && span_is_seq(net, first, last)) return true;
     if (!span_is_chain(net, first, last)) return false;
     if (net->opt_group_kernel == 1) return true;
+    const int n = static_cast<int>(net->layers.size());
+    for (int i = first; i <= last; i++)
+        if (i + 1 < n && net->layers[i + 1].d.op == DLF_DWCONV && net->layers[i + 1].d.src == i) return false;
     const ChainTiling t = chain_tc_tiling(chain_args(net, first, last, nullptr, nullptr), s_max, s_max);
     if (!t.ok) return false;
     double single_us = 0.0;
@@ -428,9 +433,9 @@ static bool tuner_may_fuse(const dlf_net* net, int first, int last, bool prefix,
         const Layer& l = net->layers[i];
         const double bytes = static_cast<double>(l.in[0] * l.in[1] * l.in[2] * l.in[3] * 2) + static_cast<double>(l.bytes) + static_cast<double>(l.w_elems * 2) +
                              (l.d.res_src != -2 ? static_cast<double>(l.bytes) : 0.0);
-        single_us += std::max(static_cast<double>(l.flops) / 600e6, bytes / 5.5e6) + 5.5;
+        single_us += std::max(static_cast<double>(l.flops) / 600e6, bytes / 5.5e6) + 7.0;
     }
-    return t.cost / 1.9e3 < single_us;
+    return t.cost / 1.9e3 + 5.5 < 0.9 * single_us;
 }
 
 static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* final_out, cudaStream_t s) {

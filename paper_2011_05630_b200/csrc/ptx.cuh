@@ -81,10 +81,11 @@ constexpr uint64_t kWaitLimitNs = 1000000000ull;  // one second
 // giving up, `code` (which wait, which CTA) is stored in the global status word.  HOT marks the waits on
 // the critical path between two layers of a fused group: they keep polling much longer before they
 // start to sleep.  (try_wait with a suspend-time hint instead of this loop was measured 1-3 % slower.)
-template <bool HOT = false>
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status, int code, uint64_t limit_ns = kWaitLimitNs) {
-    if (mbar_try_wait(bar, parity)) return true;
+// The polling loop is a function of its own (one copy per kernel instead of one per wait site: a kernel has dozens of
+// waits, and their inlined loops made up a large part of its code); the first poll, which usually succeeds, stays inline.
+template <bool HOT>
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status, int code,
+                                            uint64_t limit_ns) {
     uint64_t t0 = 0;   // the global timer is read only once a wait has lasted a while
     uint32_t spins = 0;
     while (true) {
@@ -102,6 +103,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
             }
         }
     }
+}
+template <bool HOT = false>
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status, int code, uint64_t limit_ns = kWaitLimitNs) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow<HOT>(bar, parity, abort_flag, status, code, limit_ns);
 }
 
 // Warp-wide form: every lane polls (a whole warp stays on the issue path so that the addresses it

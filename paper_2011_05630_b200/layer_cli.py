@@ -1,4 +1,6 @@
-"""Runs one convolution layer a few times through the C ABI (for profiler captures and quick checks).
+"""Command line for one layer: builds a single convolution / depthwise / max-pool layer, or one fused inverted-residual
+block, with the seeded synthetic tensors of the workloads, runs it a few times through the C ABI and prints which kernel
+ran (handy under a profiler, or to try a shape before putting it into a network).
 
     python -m paper_2011_05630_b200.layer_cli N H W CIN COUT K [--as-chain] [--reps 3] [--stride 1]
                                               [--op conv|dwconv|maxpool] [--mbconv HID]
@@ -9,8 +11,6 @@ inverted-residual block CIN -> HID (1x1) -> depthwise 3x3 (--stride) -> COUT (1x
 from __future__ import annotations
 
 import argparse
-
-import numpy as np
 
 
 def main():
@@ -34,16 +34,9 @@ def main():
                   mk("conv", a.mbconv, a.cout, 1, 1, 1, "none", res)]
     else:
         layers = [mk(a.op, a.cin, a.cin if a.op != "conv" else a.cout, a.k, a.stride, -1, "none" if a.op == "maxpool" else "relu")]
-    rng = np.random.default_rng(0)
-    params = []
-    for l in layers:
-        if l["op"] == "maxpool":
-            params.append(None)
-            continue
-        cg = l["cin"] // l["groups"]
-        params.append(((rng.standard_normal((l["cout"], l["kh"], l["kw"], cg)) * (l["kh"] * l["kw"] * cg) ** -0.5).astype(np.float16),
-                       (rng.standard_normal(l["cout"]) * 0.1).astype(np.float32)))
-    x = rng.uniform(-1, 1, (a.n, a.h, a.w, a.cin)).astype(np.float16)
+    from . import synth
+    params = synth.layer_params("layer_cli", layers)
+    x = synth.network_input("layer_cli", a.n, a.h, a.w, a.cin)
     sess = Session(layers, params, a.n, a.h, a.w, a.cin)
     xd = sess.upload(x)
     B.net_set_option(sess.net, B.OPT_CUDA_GRAPH, 0)
