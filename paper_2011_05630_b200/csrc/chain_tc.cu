@@ -254,6 +254,42 @@ __device__ __forceinline__ void epi_last(const ChainParams& p, const ChainLayerP
     }
 }
 
+// The UMMAs of one pass whose operands are all in shared memory already (resident weights; an operand tile of the group,
+// or a resident input frame): for every 64-channel chunk, every tap, every block of the pass, four K = 16 steps.  The
+// issuing warp is bound by its own instruction stream (measured: about 4 cycles per instruction, and a pass of 36 UMMAs
+// cost it 3000 instructions in the general loop below), so this path is kept to a few instructions per UMMA: 32-bit
+// descriptor words, the tap loop unrolled at compile time, nothing but adds inside.
+//   a16 / b16: low descriptor words of tap (0, 0), chunk 0, block 0 / of the first weight slab
+template <int K>
+__device__ __forceinline__ void issue_pass_resident(uint32_t d0, uint32_t slot_cols, int nblk, uint32_t a16, uint32_t a_chunk16, uint32_t b16,
+                                                    uint32_t w_tap16, uint32_t idesc, int kchunks, int ksteps_last, int pitch) {
+#pragma unroll 1
+    for (int kc = 0; kc < kchunks; kc++, a16 += a_chunk16) {
+        const bool whole = kc + 1 < kchunks || ksteps_last == 4;
+#pragma unroll
+        for (int r = 0; r < K; r++) {
+#pragma unroll
+            for (int sx = 0; sx < K; sx++) {
+                uint32_t a = a16 + static_cast<uint32_t>((r * pitch + sx) * 8), d = d0;
+                const uint32_t acc = (kc | r | sx) != 0;
+#pragma unroll 1
+                for (int blk = 0; blk < nblk; blk++, a += (128 * 128) >> 4, d += slot_cols) {
+                    if (elect_one()) {
+                        if (whole) {
+                            umma_f16_x4(d, a, b16, idesc, acc);
+                        } else {
+                            umma_f16_lo(d, a, kDescHiSw128, b16, idesc, acc);
+                            if (ksteps_last > 1) umma_f16_lo(d, a + 2, kDescHiSw128, b16 + 2, idesc, 1);
+                            if (ksteps_last > 2) umma_f16_lo(d, a + 4, kDescHiSw128, b16 + 4, idesc, 1);
+                        }
+                    }
+                }
+                b16 += w_tap16;
+            }
+        }
+    }
+}
+
 template <int OUT_MODE>
 __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_constant__ ChainParams p) {
     extern __shared__ uint8_t smem_raw[];
@@ -464,83 +500,132 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                         tc_fence_after_sync();
                         const uint32_t d_tmem0 = tmem_base + col0 + half * half_cols;
                         const uint32_t row0 = (qs + static_cast<uint32_t>(b0) * 128u) * 128u;
-                        int r0 = 0, sx0 = 0;   // kernel row / column of tap t0
+                        if (w_res && !(l == 0 && in_ring)) {
+                            // ---- the lean path: every operand of the pass is in shared memory ----------------------
+                            if (l == 0 && first_pass) {   // the tile's input frame has landed
 #pragma unroll 1
-                        for (int t0 = 0; t0 < taps && ok; t0 += tg) {
+                                for (int kc = 0; kc < kchunks && ok; kc++)
+                                    ok = mbar_wait_warp<true>(&in_full_bar[in_rd * in_group + kc], in_ph, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
+                                if (!ok) break;
+                                DLF_TRACE_ACC(tacc, 0, tmark);
+                            }
+                            const uint32_t a_base = l == 0 ? in_base + static_cast<uint32_t>(in_rd * in_group) * in_slot_bytes : abuf;
+                            const uint32_t a_chunk16 = (l == 0 ? in_slot_bytes : aplane_bytes) >> 4;
+                            const uint32_t a16 = umma_desc_lo(a_base + row0) - static_cast<uint32_t>(pad * (pitch + 1) * 8);
+                            const uint32_t b16 = umma_desc_lo(w_res0) + static_cast<uint32_t>(c * kchunks * taps) * w_tap16;
+                            if (k == 3) issue_pass_resident<3>(d_tmem0, slot_cols, nblk, a16, a_chunk16, b16, w_tap16, idesc, kchunks, ksteps_last, pitch);
+                            else issue_pass_resident<1>(d_tmem0, slot_cols, nblk, a16, a_chunk16, b16, w_tap16, idesc, kchunks, ksteps_last, pitch);
+                            DLF_TRACE_ACC(tacc, 4, tmark);
+                            if (elect_one()) umma_commit(&acc_full_bar[region * 2 + half]);
+                            __syncwarp();
+                            first_pass = false;
+                            continue;
+                        }
+                        if (w_res && l == 0 && in_ring) {
+                            // ---- lean path of a 1x1 first layer whose input planes stream through the slots ----------
+                            uint32_t b16 = umma_desc_lo(w_res0) + static_cast<uint32_t>(c * kchunks) * w_tap16;
 #pragma unroll 1
-                            for (int g0 = 0; g0 < kchunks; g0 += kg) {
-                                const int g_end = min(kg, kchunks - g0);
-                                if (l == 0 && (in_ring || (first_pass && t0 == 0))) {   // the planes this step reads have landed
-                                    int rd = in_rd, j = in_ring ? in_j : g0;
-                                    uint32_t ph = in_ph;
+                            for (int kc = 0; kc < kchunks && ok; kc++, b16 += w_tap16) {
+                                const int in_slot = in_rd * in_group + in_j;
+                                ok = mbar_wait_warp<true>(&in_full_bar[in_slot], in_ph, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
+                                if (!ok) break;
+                                uint32_t a = umma_desc_lo(in_base + static_cast<uint32_t>(in_slot) * in_slot_bytes + row0), d = d_tmem0;
+                                const bool whole = kc + 1 < kchunks || ksteps_last == 4;
 #pragma unroll 1
-                                    for (int g = 0; g < g_end && ok; g++) {
-                                        ok = mbar_wait_warp<true>(&in_full_bar[rd * in_group + j], ph, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
-                                        if (++j == in_group) { j = 0; if (++rd == ring_rounds) { rd = 0; ph ^= 1u; } }
+                                for (int blk = 0; blk < nblk; blk++, a += (128 * 128) >> 4, d += slot_cols) {
+                                    if (elect_one()) {
+                                        if (whole) {
+                                            umma_f16_x4(d, a, b16, idesc, kc != 0);
+                                        } else {
+                                            umma_f16_lo(d, a, kDescHiSw128, b16, idesc, kc != 0);
+                                            if (ksteps_last > 1) umma_f16_lo(d, a + 2, kDescHiSw128, b16 + 2, idesc, 1);
+                                            if (ksteps_last > 2) umma_f16_lo(d, a + 4, kDescHiSw128, b16 + 4, idesc, 1);
+                                        }
                                     }
-                                    if (!ok) break;
-                                    DLF_TRACE_ACC(tacc, 0, tmark);
                                 }
-                                if (!w_res) {
+                                if (elect_one()) umma_commit(&in_empty_bar[in_slot]);   // the plane is free once these have read it
+                                if (++in_j == in_group) { in_j = 0; if (++in_rd == ring_rounds) { in_rd = 0; in_ph ^= 1u; } }
+                            }
+                            if (!ok) break;
+                            DLF_TRACE_ACC(tacc, 4, tmark);
+                            if (elect_one()) umma_commit(&acc_full_bar[region * 2 + half]);
+                            __syncwarp();
+                            first_pass = false;
+                            continue;
+                        }
+                        // ---- weights streamed through the ring: one box = tg taps x kg chunks, waited for and released as a whole ----
+                        {
+                            const uint32_t a_base = l == 0 ? in_base + static_cast<uint32_t>(in_rd * in_group) * in_slot_bytes : abuf;
+                            const uint32_t a_chunk16 = (l == 0 ? in_slot_bytes : aplane_bytes) >> 4;
+                            const uint32_t a16 = umma_desc_lo(a_base + row0) - static_cast<uint32_t>(pad * (pitch + 1) * 8);
+                            const bool a_ring = l == 0 && in_ring;   // (then k == 1: the planes come through the slots one by one)
+                            if (l == 0 && !in_ring && first_pass) {   // the tile's input frame has landed
+#pragma unroll 1
+                                for (int kc = 0; kc < kchunks && ok; kc++)
+                                    ok = mbar_wait_warp<true>(&in_full_bar[in_rd * in_group + kc], in_ph, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
+                                if (!ok) break;
+                                DLF_TRACE_ACC(tacc, 0, tmark);
+                            }
+                            int r0 = 0, sx0 = 0;   // kernel row / column of tap t0
+#pragma unroll 1
+                            for (int t0 = 0; t0 < taps && ok; t0 += tg) {
+#pragma unroll 1
+                                for (int g0 = 0; g0 < kchunks && ok; g0 += kg) {
                                     ok = mbar_wait_warp<true>(&wfull_bar[w_st], w_ph, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
                                     if (!ok) break;
                                     DLF_TRACE_ACC(tacc, 3, tmark);
-                                }
-                                // Descriptors as 32-bit low words (start address in 16-byte units; the high word is a constant): every value
-                                // below is warp-uniform, the whole warp walks the loops and one elected lane issues.
-                                uint32_t b_lo = umma_desc_lo(w_res ? w_res0 + static_cast<uint32_t>((c * kchunks + g0) * taps + t0) * (w_tap16 << 4)
-                                                                   : base + p.ring_off + w_st * p.stage_bytes);
-                                {
-                                    int rd = in_rd, j = in_ring ? in_j : g0;
+                                    uint32_t b16 = umma_desc_lo(base + p.ring_off + w_st * p.stage_bytes);
+                                    const int g_end = min(kg, kchunks - g0);
 #pragma unroll 1
-                                    for (int g = 0; g < g_end; g++) {
+                                    for (int g = 0; g < g_end && ok; g++) {
                                         const int kc = g0 + g;
-                                        const int ksteps = (kc == kchunks - 1) ? ksteps_last : 4;
-                                        uint32_t aplane;
-                                        const int in_slot = rd * in_group + j;
-                                        if (l == 0) {
-                                            aplane = in_base + in_slot * in_slot_bytes + row0;
-                                            if (++j == in_group) { j = 0; if (++rd == ring_rounds) rd = 0; }
+                                        const bool whole = kc + 1 < kchunks || ksteps_last == 4;
+                                        uint32_t a_kc;
+                                        int in_slot = 0;
+                                        if (a_ring) {
+                                            in_slot = in_rd * in_group + in_j;
+                                            ok = mbar_wait_warp<true>(&in_full_bar[in_slot], in_ph, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
+                                            if (!ok) break;
+                                            a_kc = umma_desc_lo(in_base + static_cast<uint32_t>(in_slot) * in_slot_bytes + row0);
                                         } else {
-                                            aplane = abuf + kc * aplane_bytes + row0;
+                                            a_kc = a16 + static_cast<uint32_t>(kc) * a_chunk16;
                                         }
-                                        const uint32_t a_kc = umma_desc_lo(aplane);
-                                        int shift16 = ((r0 - pad) * pitch + (sx0 - pad)) * 8;   // tap's row shift in 16-byte units
+                                        uint32_t shift16 = static_cast<uint32_t>((r0 * pitch + sx0) * 8);
                                         int sx = sx0;
                                         uint32_t acc = (r0 | sx0 | kc) != 0;
 #pragma unroll 1
-                                        for (int tt = 0; tt < tg; tt++, b_lo += w_tap16) {
-                                            uint32_t a_lo = a_kc + shift16, d_tmem = d_tmem0;
+                                        for (int tt = 0; tt < tg; tt++, b16 += w_tap16) {
+                                            uint32_t a = a_kc + shift16, d = d_tmem0;
 #pragma unroll 1
-                                            for (int b = 0; b < nblk; b++, d_tmem += slot_cols, a_lo += (128 * 128) >> 4) {
+                                            for (int blk = 0; blk < nblk; blk++, a += (128 * 128) >> 4, d += slot_cols) {
                                                 if (elect_one()) {
-                                                    umma_f16_lo(d_tmem, a_lo, kDescHiSw128, b_lo, idesc, acc);
-                                                    if (ksteps > 1) umma_f16_lo(d_tmem, a_lo + 2, kDescHiSw128, b_lo + 2, idesc, 1);
-                                                    if (ksteps > 2) umma_f16_lo(d_tmem, a_lo + 4, kDescHiSw128, b_lo + 4, idesc, 1);
-                                                    if (ksteps > 3) umma_f16_lo(d_tmem, a_lo + 6, kDescHiSw128, b_lo + 6, idesc, 1);
+                                                    if (whole) {
+                                                        umma_f16_x4(d, a, b16, idesc, acc);
+                                                    } else {
+                                                        umma_f16_lo(d, a, kDescHiSw128, b16, idesc, acc);
+                                                        if (ksteps_last > 1) umma_f16_lo(d, a + 2, kDescHiSw128, b16 + 2, idesc, 1);
+                                                        if (ksteps_last > 2) umma_f16_lo(d, a + 4, kDescHiSw128, b16 + 4, idesc, 1);
+                                                    }
                                                 }
                                             }
                                             acc = 1;
                                             shift16 += 8;
-                                            if (++sx == k) { sx = 0; shift16 += (pitch - k) * 8; }
+                                            if (++sx == k) { sx = 0; shift16 += static_cast<uint32_t>((pitch - k) * 8); }
                                         }
-                                        // a streamed input plane is free again once these instructions have read it
-                                        if (l == 0 && in_ring && elect_one()) umma_commit(&in_empty_bar[in_slot]);
+                                        if (a_ring) {   // the plane is free once these have read it
+                                            if (elect_one()) umma_commit(&in_empty_bar[in_slot]);
+                                            if (++in_j == in_group) { in_j = 0; if (++in_rd == ring_rounds) { in_rd = 0; in_ph ^= 1u; } }
+                                        }
                                     }
-                                    if (!w_res && elect_one()) umma_commit(&wempty_bar[w_st]);
+                                    if (!ok) break;
+                                    if (elect_one()) umma_commit(&wempty_bar[w_st]);
+                                    __syncwarp();
+                                    if (++w_st == stages) { w_st = 0; w_ph ^= 1u; }
+                                    DLF_TRACE_ACC(tacc, 4, tmark);
                                 }
-                                __syncwarp();
-                                if (!w_res && ++w_st == stages) { w_st = 0; w_ph ^= 1u; }
-                                if (l == 0 && in_ring) {   // the streamed planes of this step are consumed
-                                    in_j += g_end;
-#pragma unroll 1
-                                    while (in_j >= in_group) { in_j -= in_group; if (++in_rd == ring_rounds) { in_rd = 0; in_ph ^= 1u; } }
-                                }
-                                DLF_TRACE_ACC(tacc, 4, tmark);
+                                sx0 += tg;
+                                while (sx0 >= k) { sx0 -= k; r0++; }
                             }
-                            sx0 += tg;
-#pragma unroll 1
-                            while (sx0 >= k) { sx0 -= k; r0++; }
                         }
                         if (ok && elect_one()) umma_commit(&acc_full_bar[region * 2 + half]);
                         __syncwarp();
@@ -1032,14 +1117,14 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
                         if (y.stg_bufs == 0 && oc.mode == OUT_STAGE) break;   // not stageable at this tile size
                     }
                     if (!y.ok) continue;
-                    // Per-tile time in SM clocks, from what was measured on B200.  The issuing warp is bound by its own
-                    // instruction stream, not by the tensor core: a step (one tap group x K-chunk group of one pass) costs
-                    // it about 900 cycles plus 40 per UMMA, whatever the tensor core then needs (operand reads from shared
-                    // memory vs. math); a weight box taken from the ring adds a handshake; a layer can start about 900
-                    // cycles after its predecessor's last instruction at the earliest (commit, drain of the last pass, fences,
-                    // wake-ups); one epilogue warp turns a 128 x 32 piece of an accumulator into fp16 in 500 (operand tile)
-                    // to 1300 (staged output with a residual) cycles; the weight ring delivers its own size per TMA round
-                    // trip.
+                    // Per-tile time in SM clocks, from what was measured on B200.  Every role of this kernel is bound by
+                    // its own instruction stream (about 4 cycles per instruction of a lone warp): the issuing warp spends
+                    // about 150 cycles per weight slab group it walks (500 when the slab comes through the ring: wait,
+                    // release) plus 25 per UMMA, unless the tensor core needs longer (operand reads from shared memory vs.
+                    // math); a layer can start about 900 cycles after its predecessor's last instruction at the earliest
+                    // (commit, fences, wake-ups) plus the drain of the last pass; a pair of epilogue warps turns a 128 x 64
+                    // piece of an accumulator into fp16 in 1200 (operand tile) to 3300 (staged output with a residual)
+                    // cycles; the weight ring delivers its own size per TMA round trip.
                     double chain = 0.0, epi_last_clk = 0.0, w_bytes = 0.0, useful = 0.0, computed = 0.0, in_reloads = 1.0;
                     for (int l = 0; l < L; l++) {
                         const LayerGeom& g = y.g[l];
@@ -1055,16 +1140,16 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
                             const double straddle = (a.k[l] == 1 || g.in_dense) ? 0.0 : (pitch % 8 == 0 ? 6.0 / 9.0 : 8.0 / 9.0);
                             tensor += static_cast<double>(g.nb) * ksteps * (std::max(32.0 * (1.0 + straddle) + n / 4.0, n / 2.0) + 6.0);
                         }
-                        const double issue = boxes * (stages == 0 ? 900.0 : 1300.0) + 40.0 * g.n_chunks * g.nb * ksteps;
+                        const double issue = boxes * (stages == 0 ? 150.0 : 500.0) + 25.0 * g.n_chunks * g.nb * ksteps;
                         const double mma = std::max(issue, tensor);
                         const double units = static_cast<double>(g.nb) * ((g.n_pad + 63) / 64);   // 128 x 32 pieces per warp of a group
                         if (l < L - 1) {
                             // the next layer starts when this one's last pass has been drained and handed over
-                            const double epi = units * 500.0;
+                            const double epi = units * 1200.0;
                             chain += std::max(mma, epi * (passes - 1) / passes) + epi / passes + 900.0;
                         } else {
                             chain += mma;
-                            epi_last_clk = units * (oc.mode == OUT_DIRECT ? 3000.0 : (a.res ? 1300.0 : 1000.0)) + (oc.mode == OUT_POOL ? units * 500.0 : 0.0) + 400.0;
+                            epi_last_clk = units * (oc.mode == OUT_DIRECT ? 6500.0 : (a.res ? 3300.0 : 2600.0)) + (oc.mode == OUT_POOL ? units * 1200.0 : 0.0) + 400.0;
                         }
                         w_bytes += static_cast<double>(g.bgroups) * a.k[l] * a.k[l] * round_up(a.cin[l], 64) * g.n_pad * 2.0;
                         if (l == 0 && im.ring) in_reloads = passes;

@@ -237,13 +237,19 @@ def test_chain_with_pool_and_residual_and_channel_change():
 
 
 def test_illegal_plans_are_rejected():
-    layers = [_conv(32, 32, 3), _conv(32, 32, 3, stride=2, src=0), _conv(32, 32, 3, src=1)]
+    layers = [_conv(32, 32, 3), _conv(32, 32, 3, stride=2, pad=1, act="none", op="maxpool", src=0), _conv(32, 32, 3, src=1)]
     sess, xd, ref = _mk(layers, "illegal", 1, 16, 16, 32)
-    for ends, sm in (([2], [4]), ([0, 2, 1], [1, 1, 1]), ([0, 1], [1, 1]), ([0, 1, 2], [0, 1, 1]), ([0, 1, 2], [1, 1, 10 ** 6])):
+    # a pool inside a group; ends not increasing; the last layer not covered; SM counts out of range
+    for ends, sm in (([2], [4]), ([0, 2, 1], [1, 1, 1]), ([0, 1], [1, 1]), ([0, 1, 2], [0, 1, 1]), ([0, 1, 2], [1, 1, 10 ** 6]), ([1, 2], [4, 4])):
         with pytest.raises(B.DlfError) as e:
             B.net_set_plan(sess.net, ends, sm)
         assert e.value.status == B.E_PLAN
     G.check_plan(sess, xd, ref, [0, 1, 2], [2, 2, 2], "legal")
+    # a stride-2 layer inside a group is no chain for the shared-memory kernel, but runs handed over through L2
+    layers = [_conv(32, 32, 3), _conv(32, 32, 3, stride=2, src=0), _conv(32, 32, 3, src=1)]
+    sess, xd, ref = _mk(layers, "strided-group", 1, 16, 16, 32)
+    G.check_plan(sess, xd, ref, [2], [4], "stride 2 inside a group")
+    assert sess.kernels() == ["conv_seq"]
 
 
 # ---- fused inverted-residual blocks --------------------------------------------------------------------
