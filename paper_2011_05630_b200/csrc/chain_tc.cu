@@ -1162,7 +1162,9 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
                     // a single input frame is loaded between two tiles; a second frame / a plane ring hides the load
                     clk = (im.slots > in_planes || im.ring) ? std::max(clk, load_in) : clk + load_in + 1500.0;
                     if (oc.mode == OUT_STAGE && oc.bufs == 1) clk += 600.0;
-                    const double cost = static_cast<double>(waves) * clk + epi_last_clk + 3000.0 + (stages == 0 ? y.w_resident_bytes / 48.0 : 0.0);
+                    // (among tilings of equal time the one that recomputes less wins: it loads less and leaves SMs free)
+                    const double cost = (static_cast<double>(waves) * clk + epi_last_clk + 3000.0 + (stages == 0 ? y.w_resident_bytes / 48.0 : 0.0)) *
+                                        (1.0 + 0.01 * (computed / useful - 1.0));
                     if (!best.ok || cost < best.cost) {
                         best.th = th; best.tw = tw; best.halo = halo; best.pitch = pitch; best.rows = rows;
                         best.tiles_h = tiles_h; best.tiles_w = tiles_w; best.n_tiles = static_cast<int>(n_tiles);

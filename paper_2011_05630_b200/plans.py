@@ -29,10 +29,16 @@ def ablation_plans(net, n_layers, sms, **over):
     sm_fractions and keeps the best); 3 no fusion, every layer on its own Eq. 5 count; 4 everything fused that
     can be, all SMs; 5 Algorithm 1's blocks, all SMs; 6 Algorithm 1's blocks and SM counts.  Strategy 3 is
     Algorithm 1 with a vanishing critical operation count (every layer closes its own block), strategy 4 with an
-    unreachable one (a block closes only where it must)."""
+    unreachable one and the hand-over through L2 allowed, so that a block closes only where no fused kernel can run the
+    layers (a pooling or fully connected layer, sixteen layers reached) and not where fusing is estimated not to pay.
+    The library's choice of hand-over is set back afterwards; setting it drops the net's current plan."""
     every = list(range(n_layers))
     per_layer = tuned_plan(net, n_layers, **dict(over, op_critical=1e-30))
-    all_fused = tuned_plan(net, n_layers, **dict(over, op_critical=1e300))
+    B.net_set_option(net, B.OPT_GROUP_KERNEL, 2)
+    try:
+        all_fused = tuned_plan(net, n_layers, **dict(over, op_critical=1e300))
+    finally:
+        B.net_set_option(net, B.OPT_GROUP_KERNEL, 0)
     tuned = tuned_plan(net, n_layers, **over)
     return [("1 no fusion, 1 SM", every, [1] * n_layers),
             ("2 no fusion, best fixed S", every, None),
