@@ -400,13 +400,30 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                 const uint32_t bytes = static_cast<uint32_t>(tg * kg * L.chunk_n) * 128u;
                 const int n_boxes = L.n_chunks * (taps / tg) * (kchunks / kg);
                 mbar_expect_tx(&wres_bar[l], static_cast<uint32_t>((n_boxes - role + kWeightWarps - 1) / kWeightWarps) * bytes);
-                int turn = 0;
+                // Every CTA wants the same slabs at the same moment: each starts its round at another box, so that the
+                // requests of the 148 CTAs spread over the L2 slices instead of queueing on the same lines.
+                const int first = (static_cast<int>(blockIdx.x) * kWeightWarps) % n_boxes;
+                int turn = 0, box = 0;
 #pragma unroll 1
                 for (int c = 0; c < L.n_chunks; c++)
 #pragma unroll 1
                     for (int t0 = 0; t0 < taps; t0 += tg)
 #pragma unroll 1
-                        for (int g0 = 0; g0 < kchunks; g0 += kg) {
+                        for (int g0 = 0; g0 < kchunks; g0 += kg, box++) {
+                            if (turn == role && box >= first) {
+                                uint8_t* dst = sbase + p.ring_off + L.w_off + static_cast<size_t>((c * kchunks + g0) * taps + t0) * L.chunk_n * 128;
+                                if (rank4) tma_load_4d(dst, &p.tmw[l], &wres_bar[l], 0, c * L.chunk_n, t0, g0);
+                                else tma_load_3d(dst, &p.tmw[l], &wres_bar[l], g0 * 64, c * L.chunk_n, t0);
+                            }
+                            if (++turn == kWeightWarps) turn = 0;
+                        }
+                turn = 0, box = 0;   // ... and the boxes before its starting point afterwards
+#pragma unroll 1
+                for (int c = 0; c < L.n_chunks && box < first; c++)
+#pragma unroll 1
+                    for (int t0 = 0; t0 < taps && box < first; t0 += tg)
+#pragma unroll 1
+                        for (int g0 = 0; g0 < kchunks && box < first; g0 += kg, box++) {
                             if (turn == role) {
                                 uint8_t* dst = sbase + p.ring_off + L.w_off + static_cast<size_t>((c * kchunks + g0) * taps + t0) * L.chunk_n * 128;
                                 if (rank4) tma_load_4d(dst, &p.tmw[l], &wres_bar[l], 0, c * L.chunk_n, t0, g0);
@@ -661,6 +678,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         cx.tmem_lane = tmem_base + (static_cast<uint32_t>((warp & 3) * 32) << 16);
         uint32_t pass_i = 0;
         bool ok = nl > 1;
+        DLF_TRACE_DECL(aacc, amark);  // cycles of CTA 0's first group-A thread: 0 accumulator wait, 1 drain, 2 fences and arrivals
 #pragma unroll 1
         for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
             const int txi = t % p.tiles_w, tyi = (t / p.tiles_w) % p.tiles_h;
@@ -684,11 +702,13 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                         const uint32_t half = pass_i & 1u;
                         ok = mbar_wait<true>(&acc_full_bar[half], (pass_i >> 1) & 1u, abort_flag, p.status, 0x700 | (blockIdx.x << 12));
                         if (!ok) break;
+                        DLF_TRACE_ACC(aacc, 0, amark);
                         tc_fence_after_sync();
                         cx.b0 = b0;
                         cx.nblk = min(L.per_pass, L.nb - b0);
                         cx.tmem_col = L.col0 + half * L.half_cols;
                         epi_inner(p, L, cx);
+                        DLF_TRACE_ACC(aacc, 1, amark);
                         fence_proxy_async_smem();  // UMMA reads these rows through the async proxy
                         tc_fence_before_sync();
                         __syncwarp();
@@ -696,8 +716,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                     }
                 }
                 if (ok && lane == 0) mbar_arrive(&act_ready_bar);
+                DLF_TRACE_ACC(aacc, 2, amark);
             }
         }
+        if (et == 0) DLF_TRACE_FLUSH_AT(p.status, aacc, 16);
     } else if (warp < 2 * kEpiWarps) {
         // ---- epilogue group B: the group's last layer --------------------------------------------------------------
         const int et = threadIdx.x - 32 * kEpiWarps;
@@ -1165,6 +1187,11 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
                     // (among tilings of equal time the one that recomputes less wins: it loads less and leaves SMs free)
                     const double cost = (static_cast<double>(waves) * clk + epi_last_clk + 3000.0 + (stages == 0 ? y.w_resident_bytes / 48.0 : 0.0)) *
                                         (1.0 + 0.01 * (computed / useful - 1.0));
+#ifdef DLF_TRACE
+                    if (getenv("DLF_TILER_LIST"))
+                        fprintf(stderr, "tile %dx%d in(%d,%d,%d) out(%d,%d) stages %d waves %lld chain %.0f epi_last %.0f load_w %.0f load_in %.0f clk %.0f red %.2f cost %.0f\n", th, tw,
+                                im.ring, im.group, im.slots, oc.mode, oc.bufs, stages, waves, chain, epi_last_clk, load_w, load_in, clk, computed / useful, cost);
+#endif
                     if (!best.ok || cost < best.cost) {
                         best.th = th; best.tw = tw; best.halo = halo; best.pitch = pitch; best.rows = rows;
                         best.tiles_h = tiles_h; best.tiles_w = tiles_w; best.n_tiles = static_cast<int>(n_tiles);

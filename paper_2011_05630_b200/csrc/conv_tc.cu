@@ -212,7 +212,13 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
         {
             const int role = warp - kProdWarp0;
             const bool is_b = role >= 2;
-            if (!is_b && !grid_wait(gs, lane, abort_flag, p.status)) return;   // the input may be a layer of this launch
+            // the first work item is decoded ahead of the wait for the previous kernel: the divisions (about a hundred
+            // cycles each for a lone warp) then cost nothing on the path from that kernel's end to the first copy
+            const TileCoord c_first = decode_work<SPLIT>(p, blockIdx.x);
+            if (!is_b) {
+                pdl_wait();
+                if (!grid_wait(gs, lane, abort_flag, p.status)) return;   // the input may be a layer of this launch
+            }
             const uint32_t parity = role & 1;
             const uint32_t my_bytes = static_cast<uint32_t>(p.kg) * (is_b ? static_cast<uint32_t>(kTps * p.BN) : static_cast<uint32_t>(p.rows)) * 128u;
             uint32_t it = 0;
@@ -220,15 +226,18 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
             DLF_TRACE_DECL(pacc, pmark);  // cycles of CTA 0's producers: 0 wait for a free stage, 1 issue
             // One ring stage: K-chunk group kq of tap group tg (row mode: tap group tg = kernel row tg, its window
             // loaded once at the row's first tap).  False once a wait has given up.
-            auto load_stage = [&](const TileCoord& c, int tg, int kq) -> bool {
-                const int st = it % p.stages;
+            // (ring position and phase are kept as counters: no division on the way to a copy)
+            int ring_st = 0;
+            uint32_t ring_ph = 0;
+            auto load_stage = [&](const TileCoord& c, int tap, int r, int s, int kq) -> bool {
+                const int st = ring_st;
+                const uint32_t ph = ring_ph;
+                if (++ring_st == p.stages) { ring_st = 0; ring_ph ^= 1u; }
                 // a ring stage belongs to ONE producer warp of each kind: a warp that skipped a phase of
                 // a stage's barrier could not tell "two phases ago" from "now" by parity
                 if ((st & 1u) != parity) return true;
-                if (!mbar_wait_warp(&sm.empty_bar[st], ((it / p.stages) & 1u) ^ 1u, abort_flag, p.status, 0x100 | (blockIdx.x << 12))) return false;
+                if (!mbar_wait_warp(&sm.empty_bar[st], ph ^ 1u, abort_flag, p.status, 0x100 | (blockIdx.x << 12))) return false;
                 DLF_TRACE_ACC(pacc, 0, pmark);
-                const int tap = tg * kTps;
-                const int r = tap / p.kw, s = tap % p.kw;
                 uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
                 if (lane == 0) mbar_expect_tx(&sm.full_bar[st], my_bytes);
                 __syncwarp();
@@ -252,16 +261,23 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
             };
 #pragma unroll 1
             for (int t = blockIdx.x; t < p.n_work && ok; t += gridDim.x) {
-                const TileCoord c = decode_work<SPLIT>(p, t);
+                const TileCoord c = t == static_cast<int>(blockIdx.x) ? c_first : decode_work<SPLIT>(p, t);
                 if (SPLIT) {   // this item's share of the tile's (tap group, K-chunk group) list
                     const int l0 = c.ks * p.kgs, l1 = min(k_iters, l0 + p.kgs);
 #pragma unroll 1
-                    for (int li = l0; li < l1 && ok; li++, it++) ok = load_stage(c, li / p.kgroups, li % p.kgroups);
+                    for (int li = l0; li < l1 && ok; li++, it++) {
+                        const int tg = li / p.kgroups, tap = tg * kTps;
+                        ok = load_stage(c, tap, tap / p.kw, tap % p.kw, li - tg * p.kgroups);
+                    }
                 } else {
+                    int r = 0, s = 0;   // kernel row and column of the tap group's first tap
 #pragma unroll 1
-                    for (int tg = 0; tg < p.tgroups && ok; tg++)
+                    for (int tg = 0; tg < p.tgroups && ok; tg++) {
 #pragma unroll 1
-                        for (int kq = 0; kq < p.kgroups && ok; kq++, it++) ok = load_stage(c, tg, kq);
+                        for (int kq = 0; kq < p.kgroups && ok; kq++, it++) ok = load_stage(c, tg * kTps, r, s, kq);
+                        s += kTps;
+                        if (s >= p.kw) { s = 0; r++; }
+                    }
                 }
             }
             if (lane == 0) DLF_TRACE_FLUSH_N(p.status, pacc, 17 + 2 * role, 2);
@@ -272,7 +288,8 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
         const uint64_t desc0 = umma_desc_sw128(0);
         const uint32_t b_chunk16 = static_cast<uint32_t>(p.BN) * 8u;  // one 64-channel weight slab, in 16-byte units
         const uint32_t a_chunk16 = static_cast<uint32_t>(p.a_bytes) >> 4;  // one 64-channel slab of the tile's pixels (rows rounded up to 8)
-        uint32_t it = 0, j = 0;
+        uint32_t it = 0, j = 0, ring_ph = 0;
+        int ring_st = 0;   // ring position and phase as counters: no division in the issue loop
         bool ok = true;
         DLF_TRACE_DECL(macc, mmark);  // cycles of CTA 0's issuer: 0 accumulator wait, 1 stage wait, 2 issue
 #pragma unroll 1
@@ -291,9 +308,10 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
             }
 #pragma unroll 1
             for (int ki = 0; ki < k_end; ki++, it++) {
-                const int st = it % p.stages;
-                ok = mbar_wait_warp(&sm.full_bar[st], (it / p.stages) & 1u, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
+                const int st = ring_st;
+                ok = mbar_wait_warp(&sm.full_bar[st], ring_ph, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                 if (!ok) break;
+                if (++ring_st == p.stages) { ring_st = 0; ring_ph ^= 1u; }
                 if (it == 0 && lane == 0) DLF_TRACE_POINT(p.status, 3);
                 DLF_TRACE_ACC(macc, 1, mmark);
                 tc_fence_after_sync();
@@ -599,7 +617,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     pdl_launch_dependents();
     // everything above overlapped the previous kernel; from here on its outputs are read - except by the
     // weight producers, which only read constants and may run ahead
-    if (warp < kProdWarp0 + 2 || warp == kStoreWarp) pdl_wait();
+    if (warp < kProdWarp0 || warp == kStoreWarp) pdl_wait();   // (the input producers wait once they have decoded their first work item)
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
 
