@@ -368,6 +368,8 @@ static bool single_kind(const dlf_net* net, int i, Kind* kind) {
     return false;
 }
 
+static bool chain_pays(const dlf_net* net, int first, int last, int sms, ChainTiling* tiling);
+
 static bool make_group(const dlf_net* net, int first, int last, int sms, Group* g) {
     g->first = first; g->last = last; g->sms = sms;
     g->tiling = ChainTiling{};
@@ -391,7 +393,15 @@ static bool make_group(const dlf_net* net, int first, int last, int sms, Group* 
     const bool seq_ok = first < last && span_is_seq(net, first, last);
     bool narrow = true;
     for (int i = first; i <= last; i++) narrow = narrow && net->layers[i].d.cin <= 64 && net->layers[i].d.cout <= 64;
-    const bool want_chain = chain_ok && (first == last || net->opt_group_kernel == 1 || (net->opt_group_kernel == 0 && narrow) || !seq_ok);
+    bool want_chain = chain_ok && (first == last || net->opt_group_kernel == 1 || (net->opt_group_kernel == 0 && narrow) || !seq_ok);
+    if (chain_ok && !want_chain && net->opt_group_kernel == 0) {   // wide layers: where the estimate says the kernel pays (few tiles per SM)
+        want_chain = chain_pays(net, first, last, sms, &g->tiling);
+        if (want_chain) {
+            g->kind = K_CHAIN_TC;
+            return true;
+        }
+        g->tiling = ChainTiling{};
+    }
     if (want_chain) {
         ChainArgs a = chain_args(net, first, last, nullptr, nullptr);
         g->tiling = chain_tc_tiling(a, sms, net->dev_sms);
@@ -417,6 +427,22 @@ static bool make_group(const dlf_net* net, int first, int last, int sms, Group* 
 // that block fuses better as a whole.  Inverted-residual blocks follow the measured rule on the hidden width.  Groups
 // handed over through L2 are proposed only when the option asks for them (measured: a device-wide barrier per layer is no
 // cheaper than a kernel boundary).  `prefix`: the layers may also be the beginning of a pattern that can still grow.
+// The estimate for a dense chain handed over in shared memory: true if the fused kernel is expected to beat one kernel per
+// layer on `sms` SMs (see above).  `tiling` receives the fused kernel's tiling.
+static bool chain_pays(const dlf_net* net, int first, int last, int sms, ChainTiling* tiling) {
+    const ChainTiling t = chain_tc_tiling(chain_args(net, first, last, nullptr, nullptr), sms, net->dev_sms > 0 ? net->dev_sms : sms);
+    if (tiling) *tiling = t;
+    if (!t.ok) return false;
+    double single_us = 0.0;
+    for (int i = first; i <= last; i++) {
+        const Layer& l = net->layers[i];
+        const double bytes = static_cast<double>(l.in[0] * l.in[1] * l.in[2] * l.in[3] * 2) + static_cast<double>(l.bytes) + static_cast<double>(l.w_elems * 2) +
+                             (l.d.res_src != -2 ? static_cast<double>(l.bytes) : 0.0);
+        single_us += std::max(static_cast<double>(l.flops) / 600e6, bytes / 5.5e6) + 7.0;
+    }
+    return t.cost / 1.9e3 + 5.5 < 0.85 * single_us;
+}
+
 static bool tuner_may_fuse(const dlf_net* net, int first, int last, bool prefix, int s_max) {
     if (first == last) return true;
     if (net->opt_no_tc) return false;
@@ -427,16 +453,7 @@ static bool tuner_may_fuse(const dlf_net* net, int first, int last, bool prefix,
     const int n = static_cast<int>(net->layers.size());
     for (int i = first; i <= last; i++)
         if (i + 1 < n && net->layers[i + 1].d.op == DLF_DWCONV && net->layers[i + 1].d.src == i) return false;
-    const ChainTiling t = chain_tc_tiling(chain_args(net, first, last, nullptr, nullptr), s_max, s_max);
-    if (!t.ok) return false;
-    double single_us = 0.0;
-    for (int i = first; i <= last; i++) {
-        const Layer& l = net->layers[i];
-        const double bytes = static_cast<double>(l.in[0] * l.in[1] * l.in[2] * l.in[3] * 2) + static_cast<double>(l.bytes) + static_cast<double>(l.w_elems * 2) +
-                             (l.d.res_src != -2 ? static_cast<double>(l.bytes) : 0.0);
-        single_us += std::max(static_cast<double>(l.flops) / 600e6, bytes / 5.5e6) + 7.0;
-    }
-    return t.cost / 1.9e3 + 5.5 < 0.85 * single_us;
+    return chain_pays(net, first, last, s_max, nullptr);
 }
 
 static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* final_out, cudaStream_t s) {

@@ -62,7 +62,7 @@ constexpr int kInputWarp = kWeightWarp0 + kWeightWarps;  // warp 21
 constexpr int kStoreWarp = kInputWarp + 1;               // warp 22
 constexpr int kThreads = 32 * (kStoreWarp + 1);
 constexpr int kWeightOpBytes = 16 * 1024;      // target size of one weight TMA box
-constexpr int kMaxSmem = 232448 - 1024;        // dynamic part: the 227 KB per-CTA limit minus the static barriers
+constexpr int kMaxSmem = 232448 - 2048;        // dynamic part: the 227 KB per-CTA limit minus the static barriers and layer table
 constexpr int kMaxBias = 4096;                 // floats of bias staged in shared memory (all layers)
 constexpr int kMaxInSlots = 16;
 constexpr int kMaxStages = 8;
@@ -298,6 +298,9 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     __shared__ uint64_t act_ready_bar, stg_full_bar[2], stg_free_bar[2], wres_bar[kMaxChain];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    // The layers' parameters, copied out of the kernel's parameter block: every role walks the layers of every tile, and
+    // a dynamically indexed read of the parameter block cost the issuing warp about 700 cycles per layer (measured).
+    __shared__ __align__(16) ChainLayerP Ls[kMaxChain];
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sbase = smem_raw + (base - smem_u32(smem_raw));
@@ -305,9 +308,17 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     volatile int* abort_flag = &abort_s;
     const int nl = p.n_layers;
-    const ChainLayerP& LL = p.L[nl - 1];
+    {
+        const uint32_t* src = reinterpret_cast<const uint32_t*>(&p.L[0]);
+        uint32_t* dst = reinterpret_cast<uint32_t*>(&Ls[0]);
+        const int words = nl * static_cast<int>(sizeof(ChainLayerP) / 4);
+#pragma unroll 1
+        for (int i = threadIdx.x; i < words; i += kThreads) dst[i] = src[i];
+    }
+    const ChainLayerP& LL = Ls[nl - 1];
 
     if (threadIdx.x == 0) {
+        DLF_TRACE_POINT(p.status, 24);
         abort_s = 0;
 #pragma unroll 1
         for (int i = 0; i < p.stages; i++) {
@@ -360,7 +371,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
     }
     const int ring_rounds = p.in_slots / p.in_group;     // producer rounds the input slots hold
     const int rounds_per_pass = p.in_planes / p.in_group;
-    const int passes0 = p.L[0].n_chunks * p.L[0].bgroups;
+    const int passes0 = p.L[0].n_chunks * p.L[0].bgroups;   // (statically indexed: read before the copy above is visible)
 
     if (warp == kInputWarp) {
         // ---- input producer: a round = in_group planes, one lane each; a lane owns its slots ---------------
@@ -395,7 +406,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             // resident weights: every layer's slabs are loaded once, the boxes dealt out to the four producers in turn
 #pragma unroll 1
             for (int l = 0; l < nl; l++) {
-                const ChainLayerP& L = p.L[l];
+                const ChainLayerP& L = Ls[l];
                 const int taps = L.k * L.k, tg = L.tg, kg = L.kg, kchunks = L.kchunks, rank4 = L.w_rank4;
                 const uint32_t bytes = static_cast<uint32_t>(tg * kg * L.chunk_n) * 128u;
                 const int n_boxes = L.n_chunks * (taps / tg) * (kchunks / kg);
@@ -411,6 +422,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
 #pragma unroll 1
                         for (int g0 = 0; g0 < kchunks; g0 += kg, box++) {
                             if (turn == role && box >= first) {
+                                if (l == 0 && role == 0 && box == first) DLF_TRACE_POINT(p.status, 25);
                                 uint8_t* dst = sbase + p.ring_off + L.w_off + static_cast<size_t>((c * kchunks + g0) * taps + t0) * L.chunk_n * 128;
                                 if (rank4) tma_load_4d(dst, &p.tmw[l], &wres_bar[l], 0, c * L.chunk_n, t0, g0);
                                 else tma_load_3d(dst, &p.tmw[l], &wres_bar[l], g0 * 64, c * L.chunk_n, t0);
@@ -440,7 +452,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
 #pragma unroll 1
                 for (int l = 0; l < nl && ok; l++) {
-                    const ChainLayerP& L = p.L[l];
+                    const ChainLayerP& L = Ls[l];
                     const uint32_t bytes = static_cast<uint32_t>(L.tg * L.kg * L.chunk_n) * 128u;  // the whole box
                     const int taps = L.k * L.k, tg = L.tg, kg = L.kg, kchunks = L.kchunks, rank4 = L.w_rank4;
 #pragma unroll 1
@@ -480,7 +492,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         for (int t = blockIdx.x; t < p.n_tiles && ok; t += gridDim.x) {
 #pragma unroll 1
             for (int l = 0; l < nl && ok; l++) {
-                const ChainLayerP& L = p.L[l];
+                const ChainLayerP& L = Ls[l];
                 const int region = (l == nl - 1) ? 1 : 0;
                 if (l > 0) {  // group A has written all of the previous layer's tile
                     ok = mbar_wait_warp<true>(&act_ready_bar, act_ph, abort_flag, p.status, 0x400 | (blockIdx.x << 12));
@@ -498,6 +510,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                 if (w_res) {   // this layer's resident weights have landed (true at once from the second tile on)
                     ok = mbar_wait_warp<true>(&wres_bar[l], 0u, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
                     if (!ok) break;
+                    if (l == 0 && t == static_cast<int>(blockIdx.x) && lane == 0) DLF_TRACE_POINT(p.status, 26);
                     DLF_TRACE_ACC(tacc, 3, tmark);
                 }
                 const uint32_t w_res0 = base + p.ring_off + L.w_off;
@@ -524,6 +537,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
                                 for (int kc = 0; kc < kchunks && ok; kc++)
                                     ok = mbar_wait_warp<true>(&in_full_bar[in_rd * in_group + kc], in_ph, abort_flag, p.status, 0x300 | (blockIdx.x << 12));
                                 if (!ok) break;
+                                if (t == static_cast<int>(blockIdx.x) && lane == 0) DLF_TRACE_POINT(p.status, 27);
                                 DLF_TRACE_ACC(tacc, 0, tmark);
                             }
                             const uint32_t a_base = l == 0 ? in_base + static_cast<uint32_t>(in_rd * in_group) * in_slot_bytes : abuf;
@@ -667,7 +681,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
         // wait for these loads
 #pragma unroll 1
         for (int l = 0; l < nl - 1; l++) {
-            const ChainLayerP& L = p.L[l];
+            const ChainLayerP& L = Ls[l];
 #pragma unroll 1
             for (int i = et; i < L.n_pad; i += 32 * kEpiWarps) bias_s[L.bias_off + i] = i < L.cout ? __ldg(L.bias + i) : 0.0f;
         }
@@ -687,7 +701,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_tc_kernel(const __grid_cons
             cx.n = t / (p.tiles_w * p.tiles_h);
 #pragma unroll 1
             for (int l = 0; l < nl - 1 && ok; l++) {
-                const ChainLayerP& L = p.L[l];
+                const ChainLayerP& L = Ls[l];
                 cx.obuf = sbase + p.act_off[l & 1];
                 cx.oplane = p.act_plane_bytes[l & 1];
                 cx.bl = bias_s + L.bias_off;
@@ -1141,8 +1155,9 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
                     if (!y.ok) continue;
                     // Per-tile time in SM clocks, from what was measured on B200.  Every role of this kernel is bound by
                     // its own instruction stream (about 4 cycles per instruction of a lone warp): the issuing warp spends
-                    // about 150 cycles per weight slab group it walks (500 when the slab comes through the ring: wait,
-                    // release) plus 25 per UMMA, unless the tensor core needs longer (operand reads from shared memory vs.
+                    // about 150 cycles per weight slab group it walks (1500 when the slab comes through the ring: measured on
+                    // ResNet bottleneck spans, where a ring of four to six boxes runs dry and every box then costs most of a
+                    // TMA round trip - the same spans run 1.3 to 1.7 times faster with resident weights) plus 25 per UMMA, unless the tensor core needs longer (operand reads from shared memory vs.
                     // math); a layer can start about 900 cycles after its predecessor's last instruction at the earliest
                     // (commit, fences, wake-ups) plus the drain of the last pass; a pair of epilogue warps turns a 128 x 64
                     // piece of an accumulator into fp16 in 1200 (operand tile) to 3300 (staged output with a residual)
@@ -1162,7 +1177,7 @@ ChainTiling chain_tc_tiling(const ChainArgs& a, int sm_count, int device_sms) {
                             const double straddle = (a.k[l] == 1 || g.in_dense) ? 0.0 : (pitch % 8 == 0 ? 6.0 / 9.0 : 8.0 / 9.0);
                             tensor += static_cast<double>(g.nb) * ksteps * (std::max(32.0 * (1.0 + straddle) + n / 4.0, n / 2.0) + 6.0);
                         }
-                        const double issue = boxes * (stages == 0 ? 150.0 : 500.0) + 25.0 * g.n_chunks * g.nb * ksteps;
+                        const double issue = boxes * (stages == 0 ? 150.0 : 1500.0) + 25.0 * g.n_chunks * g.nb * ksteps;
                         const double mma = std::max(issue, tensor);
                         const double units = static_cast<double>(g.nb) * ((g.n_pad + 63) / 64);   // 128 x 32 pieces per warp of a group
                         if (l < L - 1) {

@@ -47,6 +47,7 @@ constexpr int kEpiParts = 4;                // epilogue warps per TMEM lane quar
 constexpr int kEpiWarps = 4 * kEpiParts;
 constexpr int kMmaWarp = kEpiWarps;         // warps 0..15 epilogue (warp & 3 = TMEM lane quarter), then the UMMA issuer,
 constexpr int kProdWarp0 = kEpiWarps + 1;   // four producers: A even / A odd / B even / B odd ring stages,
+constexpr int kMaxOutBufs = 4;               // staging buffers of finished tiles
 constexpr int kStoreWarp = kProdWarp0 + 4;  // and one warp for the TMA stores of finished tiles and the TMA loads of residual tiles
 constexpr int kThreads = 32 * (kEpiWarps + 6);
 constexpr int kABytes = 128 * 128;  // 128 pixels x 64 fp16
@@ -63,6 +64,7 @@ struct ConvTcParams {
     int tps, tgroups;          // taps per ring stage (3 = a whole kernel row, see the row mode) and tap groups per K-chunk group
     int kg, kgroups, grouped;  // K chunks per ring stage; stages per tap; 1 = 5-d / 4-d maps (cin % 64 == 0)
     int stages;
+    int store_depth;              // TMA stores of finished tiles in flight (1 .. out_bufs)
     int n_work;
     int stage_out_off, bias_off;  // byte offsets in dynamic shared memory
     int out_bufs, out_buf_bytes;  // staging buffers (1 or 2) and the size of one
@@ -178,29 +180,41 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
 #pragma unroll 1
                 for (int jj = 0; jj < p.out_bufs; jj++)
                     if (static_cast<int>(blockIdx.x) + jj * static_cast<int>(gridDim.x) < p.n_work) fetch_residual(blockIdx.x + jj * gridDim.x, jj);
-            uint32_t j = 0;
+            // Up to `store_depth` stores are in flight: a store takes about 1.5 us from its issue until it has read its
+            // buffer whatever its size (measured), so a layer of short tiles (one or two loads each) that waited for
+            // every store before the next was bound by that latency, not by any bandwidth.  Every lane commits a group
+            // per tile (an empty one where it has no plane), so all lanes count the same groups.
+            const int depth = p.store_depth, bufs = p.out_bufs;
+            int b = 0, fb = 0;                // staging buffer of tile j / of the oldest store in flight
+            uint32_t ph = 0;                  // phase of sfull[b]
+            int t_free = blockIdx.x, j = 0;   // tile of the oldest store in flight
             DLF_TRACE_DECL(sacc, smark);  // cycles of CTA 0's store warp: 0 wait for a staged tile, 1 store and its read, 2 residual fetch
 #pragma unroll 1
             for (int t = blockIdx.x; t < p.n_work; t += gridDim.x, j++) {
-                const uint32_t b = j % p.out_bufs, ph = (j / p.out_bufs) & 1u;
                 if (!mbar_wait_warp(&sm.sfull_bar[b], ph, abort_flag, p.status, 0x500 | (blockIdx.x << 12))) break;
                 DLF_TRACE_ACC(sacc, 0, smark);
                 const TileCoord c = decode_work(p, t);
-                if (lane < planes_of(c)) {
+                if (lane < planes_of(c))
                     tma_store_4d(tmy_p, stage_out + b * p.out_buf_bytes + lane * kABytes, c.co0 + lane * 64, c.wo0, c.ho0, c.n0);
-                    tma_store_commit();
-                    tma_store_wait_read();  // the plane has been read: it may take the next residual / the next tile
+                tma_store_commit();
+                if (++b == bufs) { b = 0; ph ^= 1u; }
+                if (j + 1 >= depth) {
+                    tma_store_wait_read_n(depth - 1);  // the oldest store has read its buffer: it may take the next residual / tile
+                    __syncwarp();
+                    DLF_TRACE_ACC(sacc, 1, smark);
+                    const int t2 = t_free + bufs * static_cast<int>(gridDim.x);
+                    if (RES) {
+                        if (t2 < p.n_work) fetch_residual(t2, fb);
+                    } else if (lane == 0) {
+                        mbar_arrive(&sm.sfree_bar[fb]);
+                    }
+                    if (++fb == bufs) fb = 0;
+                    t_free += gridDim.x;
+                    DLF_TRACE_ACC(sacc, 2, smark);
                 }
-                __syncwarp();
-                DLF_TRACE_ACC(sacc, 1, smark);
-                const int t2 = t + p.out_bufs * static_cast<int>(gridDim.x);
-                if (RES) {
-                    if (t2 < p.n_work) fetch_residual(t2, b);
-                } else if (lane == 0) {
-                    mbar_arrive(&sm.sfree_bar[b]);
-                }
-                DLF_TRACE_ACC(sacc, 2, smark);
             }
+            tma_store_wait_read();   // shared memory outlives every store that reads it
+            __syncwarp();
             if (lane == 0) DLF_TRACE_FLUSH_N(p.status, sacc, 11, 3);
         }
     } else if (warp >= kProdWarp0) {
@@ -215,6 +229,7 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
             // the first work item is decoded ahead of the wait for the previous kernel: the divisions (about a hundred
             // cycles each for a lone warp) then cost nothing on the path from that kernel's end to the first copy
             const TileCoord c_first = decode_work<SPLIT>(p, blockIdx.x);
+            if (role == 0 && lane == 0 && gs.counter == nullptr) DLF_TRACE_POINT(p.status, 25);
             if (!is_b) {
                 pdl_wait();
                 if (!grid_wait(gs, lane, abort_flag, p.status)) return;   // the input may be a layer of this launch
@@ -238,6 +253,7 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
                 if ((st & 1u) != parity) return true;
                 if (!mbar_wait_warp(&sm.empty_bar[st], ph ^ 1u, abort_flag, p.status, 0x100 | (blockIdx.x << 12))) return false;
                 DLF_TRACE_ACC(pacc, 0, pmark);
+                if (it == 0 && role == 0 && lane == 0 && gs.counter == nullptr) DLF_TRACE_POINT(p.status, 26);
                 uint8_t* sa = stage0 + static_cast<size_t>(st) * stage_bytes;
                 if (lane == 0) mbar_expect_tx(&sm.full_bar[st], my_bytes);
                 __syncwarp();
@@ -371,7 +387,8 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
             for (int i = threadIdx.x; i < n_bias; i += 32 * kEpiWarps) bias_s[i] = i < p.Cout ? __ldg(p.bias + i) : 0.0f;
             asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
         }
-        uint32_t j = 0;
+        uint32_t j = 0, out_ph = 0;
+        int out_b = 0;   // staging buffer of the next tile and the phase of its barriers, as counters
         bool ok = true;
         if (RES && POOL) ok = grid_wait(gs, lane, abort_flag, p.status);   // residual read with plain loads
         DLF_TRACE_DECL(eacc, emark);  // cycles of CTA 0's first epilogue thread: 0 staging-buffer wait, 1 accumulator wait, 2 drain
@@ -469,10 +486,12 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
                 }
             };
             if (RES && POOL) res_load(part * 32, rcur, rok);
-            uint8_t* sout = stage_out + (j % p.out_bufs) * p.out_buf_bytes;
+            const int sb = out_b;   // this tile's staging buffer; the next tile takes the next one
+            const uint32_t sph = out_ph;
+            if (++out_b == p.out_bufs) { out_b = 0; out_ph ^= 1u; }
+            uint8_t* sout = stage_out + sb * p.out_buf_bytes;
             if (!POOL) {   // the staging buffer is free (first uses pass at once) / holds this tile's residual
-                const uint32_t ph = (j / p.out_bufs) & 1u;
-                ok = mbar_wait(&sm.sfree_bar[j % p.out_bufs], RES ? ph : ph ^ 1u, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
+                ok = mbar_wait(&sm.sfree_bar[sb], RES ? sph : sph ^ 1u, abort_flag, p.status, 0x600 | (blockIdx.x << 12));
                 if (!ok) break;
             }
             DLF_TRACE_ACC(eacc, 0, emark);
@@ -554,7 +573,7 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
             if (!POOL) {
                 fence_proxy_async_smem();  // the staging tile is read by the TMA unit
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.sfull_bar[j % p.out_bufs]);
+                if (lane == 0) mbar_arrive(&sm.sfull_bar[sb]);
             }
             if (j == 0 && issuer) DLF_TRACE_POINT(p.status, 6);
             DLF_TRACE_ACC(eacc, 2, emark);
@@ -568,7 +587,8 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
 __device__ __forceinline__ void conv_tc_init_bars(const ConvBars& sm, int stages, bool again) {
     if (again) {
         for (int i = 0; i < 8; i++) { mbar_inval(&sm.full_bar[i]); mbar_inval(&sm.empty_bar[i]); }
-        for (int i = 0; i < 2; i++) { mbar_inval(&sm.tfull_bar[i]); mbar_inval(&sm.tempty_bar[i]); mbar_inval(&sm.sfull_bar[i]); mbar_inval(&sm.sfree_bar[i]); }
+        for (int i = 0; i < 2; i++) { mbar_inval(&sm.tfull_bar[i]); mbar_inval(&sm.tempty_bar[i]); }
+        for (int i = 0; i < kMaxOutBufs; i++) { mbar_inval(&sm.sfull_bar[i]); mbar_inval(&sm.sfree_bar[i]); }
     }
     for (int i = 0; i < (again ? 8 : stages); i++) {
         mbar_init(&sm.full_bar[i], 2);  // the A and the B producer each arrive with their byte count
@@ -577,6 +597,8 @@ __device__ __forceinline__ void conv_tc_init_bars(const ConvBars& sm, int stages
     for (int i = 0; i < 2; i++) {
         mbar_init(&sm.tfull_bar[i], 1);
         mbar_init(&sm.tempty_bar[i], kEpiWarps);
+    }
+    for (int i = 0; i < kMaxOutBufs; i++) {
         mbar_init(&sm.sfull_bar[i], kEpiWarps);
         mbar_init(&sm.sfree_bar[i], 1);
     }
@@ -589,7 +611,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
                const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmr, const ConvTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[8], empty_bar[8], tfull_bar[2], tempty_bar[2];
-    __shared__ uint64_t sfull_bar[2], sfree_bar[2];  // staging buffer: filled by the epilogue / free again (residual landed)
+    __shared__ uint64_t sfull_bar[kMaxOutBufs], sfree_bar[kMaxOutBufs];  // staging buffer: filled by the epilogue / free again (residual landed)
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
 
@@ -666,7 +688,7 @@ __device__ __noinline__ void conv_seq_layer(const SeqLayer* Y, const ConvTcParam
 __global__ void __launch_bounds__(kThreads, 1) conv_seq_kernel(const __grid_constant__ SeqParams sp) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[8], empty_bar[8], tfull_bar[2], tempty_bar[2];
-    __shared__ uint64_t sfull_bar[2], sfree_bar[2];
+    __shared__ uint64_t sfull_bar[kMaxOutBufs], sfree_bar[kMaxOutBufs];
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     // the current layer's parameters, copied out of the kernel's parameter block: the roles read them all the time, and a
@@ -906,7 +928,8 @@ int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcL
         const int loads_min = p.tgroups * p.kchunks;
         // Two staging buffers (the stores of one tile drain while the next is written) where the ring keeps
         // three stages, or as many as the tile has loads, beside them; else one.
-        for (p.out_bufs = a.pool ? 1 : 2; p.out_bufs >= 1; p.out_bufs--) {
+        // (a layer of short tiles - one or two loads each - is bound by the latency of its stores: up to four buffers)
+        for (p.out_bufs = a.pool ? 1 : (loads_min <= 2 ? kMaxOutBufs : 2); p.out_bufs >= 1; p.out_bufs--) {
             // the UMMA always reads 128 rows of a slab (two more in the row mode): behind a shorter one it reads on
             // into whatever follows (those accumulator rows are never stored), which must still be this CTA's
             // shared memory
@@ -924,10 +947,12 @@ int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcL
             const int stage_bytes = p.kg * (p.a_bytes + b_bytes);
             p.stages = std::min(8, (budget - fixed) / stage_bytes);
             const int loads = p.tgroups * p.kgroups;
-            p.stages = std::min(p.stages, loads);
+            // (the ring runs on across work items: a tile with one or two loads still wants four stages, so that the
+            // next tiles' copies are in flight while this one is multiplied and drained)
+            p.stages = std::min(p.stages, std::max(loads, 4));
             p.stage_out_off = p.stages * stage_bytes;
             p.bias_off = p.stage_out_off + p.out_bufs * p.out_buf_bytes;
-            if (p.stages >= 1 && (p.out_bufs == 1 || p.stages >= std::min(3, loads))) break;
+            if (p.stages >= 1 && (p.out_bufs == 1 || p.stages >= std::min(3, std::max(loads, p.out_bufs)))) break;
         }
         return p.stages >= std::min(min_stages, loads_min);
     };
@@ -1039,6 +1064,8 @@ int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcL
             bias_bytes = keep_bias;
         }
     }
+    // stores in flight: all buffers but one where a buffer also has to take the next tile's residual in time
+    p.store_depth = std::max(1, a.res ? p.out_bufs - 1 : p.out_bufs);
     p.splits = splits;
     p.kgs = (p.tgroups * p.kgroups + splits - 1) / splits;
     if (splits > 1) {
