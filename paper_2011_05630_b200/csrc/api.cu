@@ -60,8 +60,8 @@ int encode_tmap(void* out_map, const void* base, int rank, const uint64_t* dims,
     return DLF_OK;
 }
 
-enum Kind { K_CHAIN_TC, K_CONV_TC, K_CONV_DIRECT, K_DW, K_FC, K_MAXPOOL, K_GAVG, K_STEM_TC, K_MBCONV, K_CONV_SEQ };
-static const char* kKindName[] = {"chain_tc", "conv_tc", "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool", "stem_tc", "mbconv_tc", "conv_seq"};
+enum Kind { K_CHAIN_TC, K_CONV_TC, K_CONV_DIRECT, K_DW, K_FC, K_MAXPOOL, K_GAVG, K_STEM_TC, K_MBCONV, K_CONV_SEQ, K_CONV_DUAL };
+static const char* kKindName[] = {"chain_tc", "conv_tc", "conv_direct", "dw3x3", "fc", "maxpool", "gavgpool", "stem_tc", "mbconv_tc", "conv_seq", "conv_tc"};
 
 struct Layer {
     dlf_layer_desc d;
@@ -317,6 +317,45 @@ static ConvArgs fc_as_conv_args(const dlf_net* net, int i, const void* in_dev, v
     return a;
 }
 
+// ---- projection branch + expansion layer of a residual block as ONE product -----------------------------------------------
+// [1x1 projection (stride 1 or 2, linear) of the block's input, 1x1 expansion of the block's 3x3 output + that projection as
+// residual]: y = act(x_e * W_e + b_e + x_p * W_p + b_p) is one implicit GEMM whose K runs over both inputs' channels, so the
+// projection's map is never written nor read back; it joins the fp32 accumulator without its own fp16 rounding (at most half
+// an fp16 unit in the last place of the projection's value away from the layer-by-layer result).
+static bool span_is_projadd(const dlf_net* net, int first, int last) {
+    if (net->opt_no_tc || last != first + 1) return false;
+    const int n = static_cast<int>(net->layers.size());
+    const dlf_layer_desc& pj = net->layers[first].d;
+    const dlf_layer_desc& ex = net->layers[last].d;
+    if (pj.op != DLF_CONV || ex.op != DLF_CONV || pj.groups != 1 || ex.groups != 1) return false;
+    if (pj.kh != 1 || pj.kw != 1 || pj.pad != 0 || pj.pool || pj.res_src != -2 || pj.act != DLF_ACT_NONE) return false;
+    if (ex.kh != 1 || ex.kw != 1 || ex.pad != 0 || ex.stride != 1 || ex.pool) return false;
+    if (ex.res_src != first || ex.src == first || ex.src >= first) return false;
+    for (int j = first + 1; j < n; j++) {   // the projection's map is used by the expansion layer's sum alone
+        const dlf_layer_desc& d = net->layers[j].d;
+        if (d.src == first || (d.res_src == first && j != last)) return false;
+    }
+    ConvArgs a = conv_args(net, last, nullptr, nullptr);
+    a.res = nullptr;
+    const Layer& pl = net->layers[first];
+    a.x2 = &a;   // only whether there is one matters here
+    a.H2 = static_cast<int>(pl.in[1]); a.W2 = static_cast<int>(pl.in[2]); a.Cin2 = pj.cin; a.stride2 = pj.stride;
+    return conv_tc_dual_supported(a);
+}
+
+static ConvArgs projadd_args(const dlf_net* net, int first, int last, const void* in_dev, void* out_dev) {
+    ConvArgs a = conv_args(net, last, in_dev, out_dev);
+    const Layer& pl = net->layers[first];
+    a.res = nullptr;
+    a.splitk_ws = nullptr;
+    a.splitk_bytes = 0;
+    a.x2 = pl.d.src < 0 ? in_dev : slot(net, pl.d.src);
+    a.w2 = pl.w;
+    a.bias2 = pl.bias;
+    a.H2 = static_cast<int>(pl.in[1]); a.W2 = static_cast<int>(pl.in[2]); a.Cin2 = pl.d.cin; a.stride2 = pl.d.stride;
+    return a;
+}
+
 // ---- groups handed over through L2 -------------------------------------------------------------------------------------
 // Any run of dense convolutions the single-layer tensor-core kernel takes (any kernel size, stride 1 or 2, fused pool,
 // residual from anywhere, a projection branch) can run as ONE persistent kernel whose CTAs walk the layers together with a
@@ -386,6 +425,10 @@ static bool make_group(const dlf_net* net, int first, int last, int sms, Group* 
         g->kind = K_MBCONV;
         return g->mb_tiling.ok;
     }
+    if (span_is_projadd(net, first, last)) {
+        g->kind = K_CONV_DUAL;
+        return true;
+    }
     // Two ways to fuse dense convolutions: hand-over in shared memory (a chain of stride-1 1x1 / 3x3 layers, tile by tile) or
     // through L2 (any run of dense convolutions, layer by layer behind a device-wide barrier).  Unless an option says
     // otherwise the first is taken for narrow layers (at most 64 channels: there it was measured faster), the second elsewhere.
@@ -448,6 +491,8 @@ static bool tuner_may_fuse(const dlf_net* net, int first, int last, bool prefix,
     if (net->opt_no_tc) return false;
     if (span_is_mbconv(net, first, last, prefix, kTunerMaxHidden)) return true;
     if (net->opt_group_kernel == 2 && span_is_seq(net, first, last)) return true;
+    // a projection and the expansion layer it is added to are one product with a longer K: never slower than the two kernels
+    if (span_is_projadd(net, first, last)) return true;
     if (!span_is_chain(net, first, last)) return false;
     if (net->opt_group_kernel == 1) return true;
     const int n = static_cast<int>(net->layers.size());
@@ -478,6 +523,7 @@ static int launch_group(dlf_net* net, const Group& g, const void* in_dev, void* 
         case K_CONV_TC:
             if (z.d.op == DLF_FC) return launch_conv_tc(fc_as_conv_args(net, g.first, in_dev, y), g.sms, status, s);
             return launch_conv_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
+        case K_CONV_DUAL: return launch_conv_tc(projadd_args(net, g.first, g.last, in_dev, y), g.sms, status, s);
         case K_STEM_TC: return launch_stem_tc(conv_args(net, g.first, in_dev, y), g.sms, status, s);
         case K_CONV_DIRECT: return launch_conv_direct(conv_args(net, g.first, in_dev, y), g.sms, s);
         case K_DW: return launch_dw3x3(conv_args(net, g.first, in_dev, y), g.sms, s);
@@ -1199,6 +1245,7 @@ int dlf_net_group_model(const dlf_net* net, int group, int64_t* flops, int64_t* 
         fl += l.flops;
         by += l.w_elems * 2 + (is_param(l) ? l.d.cout * 4 : 0);
         if (l.d.res_src != -2 && l.d.res_src < g.first) by += l.out[0] * l.ho_pre * l.wo_pre * l.out[3] * 2;
+        if (g.kind == K_CONV_DUAL && i > g.first) by += l.in[0] * l.in[1] * l.in[2] * l.in[3] * 2;   // the expansion layer's own input
         // a group handed over through L2 still writes every map to its slot and reads it back: counted like separate layers
         if (g.kind == K_CONV_SEQ) {
             if (i > g.first) by += l.in[0] * l.in[1] * l.in[2] * l.in[3] * 2;

@@ -72,7 +72,9 @@ struct ConvTcParams {
     float* partial;               // split-K: fp32 partial tiles [tile][split][row][acc_stride]
     int* counters;                // split-K: arrivals per (tile, epilogue warp); zero between launches
     uint32_t tmem_cols;
+    int kchunks1, stride2;        // second source: 64-channel chunks kchunks1 .. kchunks-1 of K come from it, read with stride2
     const float* bias;
+    const float* bias2;           // second source's bias (added to the first's), or null
     const __half* res;
     __half* out;
     int* status;
@@ -151,7 +153,8 @@ struct ConvBars {
 // its wind-down.  Called once by the single-layer kernel and once per layer by the multi-layer kernel.
 template <int ACT, bool POOL, bool RES, bool ROW, bool SPLIT>
 __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CUtensorMap* tmw_p, const CUtensorMap* tmy_p,
-                                              const CUtensorMap* tmr_p, const ConvTcParams& p, const ConvBars& sm, uint32_t tmem_base,
+                                              const CUtensorMap* tmr_p, const CUtensorMap* tmx2_p, const CUtensorMap* tmw2_p,
+                                              const ConvTcParams& p, const ConvBars& sm, uint32_t tmem_base,
                                               uint8_t* stage0, uint32_t base, const GridSync& gs) {
     float* bias_s = reinterpret_cast<float*>(stage0 + p.bias_off);
     constexpr int kTps = ROW ? 3 : 1;   // taps per ring stage: a whole kernel row in the row mode
@@ -259,14 +262,17 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
                 __syncwarp();
                 if (lane < p.kg) {   // a chunk past C_in / 64 lies outside the tensor map and arrives as zeros
                     const int kc = kq * p.kg + lane;
+                    const bool second = kc >= p.kchunks1;   // (1x1 layers with whole 64-channel chunks only: see conv_tc_dual_supported)
                     if (is_b) {
                         uint8_t* dst = sa + p.kg * p.a_bytes + lane * kTps * p.BN * 128;
-                        if (p.grouped) tma_load_4d(dst, tmw_p, &sm.full_bar[st], 0, c.co0, tap, kc);
+                        if (second) tma_load_4d(dst, tmw2_p, &sm.full_bar[st], 0, c.co0, 0, kc - p.kchunks1);
+                        else if (p.grouped) tma_load_4d(dst, tmw_p, &sm.full_bar[st], 0, c.co0, tap, kc);
                         else tma_load_3d(dst, tmw_p, &sm.full_bar[st], kc * 64, tap, c.co0);
                     } else {
                         const int wi = c.wo0 * p.stride - p.pad + s, hi = c.ho0 * p.stride - p.pad + r;
                         uint8_t* dst = sa + lane * p.a_bytes;
-                        if (p.grouped) tma_load_5d(dst, tmx_p, &sm.full_bar[st], 0, wi, hi, c.n0, kc);
+                        if (second) tma_load_5d(dst, tmx2_p, &sm.full_bar[st], 0, c.wo0 * p.stride2, c.ho0 * p.stride2, c.n0, kc - p.kchunks1);
+                        else if (p.grouped) tma_load_5d(dst, tmx_p, &sm.full_bar[st], 0, wi, hi, c.n0, kc);
                         else tma_load_4d(dst, tmx_p, &sm.full_bar[st], kc * 64, wi, hi, c.n0);
                     }
                 }
@@ -384,7 +390,7 @@ __device__ __forceinline__ void conv_tc_roles(const CUtensorMap* tmx_p, const CU
             // warps alone, after the CTA-wide barrier, so that the producers' first copies do not wait for these loads
             const int n_bias = p.n_tiles_n * p.BN;
 #pragma unroll 1
-            for (int i = threadIdx.x; i < n_bias; i += 32 * kEpiWarps) bias_s[i] = i < p.Cout ? __ldg(p.bias + i) : 0.0f;
+            for (int i = threadIdx.x; i < n_bias; i += 32 * kEpiWarps) bias_s[i] = i < p.Cout ? __ldg(p.bias + i) + (p.bias2 ? __ldg(p.bias2 + i) : 0.0f) : 0.0f;
             asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
         }
         uint32_t j = 0, out_ph = 0;
@@ -608,7 +614,8 @@ __device__ __forceinline__ void conv_tc_init_bars(const ConvBars& sm, int stages
 template <int ACT, bool POOL, bool RES, bool ROW, bool SPLIT>
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ CUtensorMap tmw,
-               const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmr, const ConvTcParams p) {
+               const __grid_constant__ CUtensorMap tmy, const __grid_constant__ CUtensorMap tmr,
+               const __grid_constant__ CUtensorMap tmx2, const __grid_constant__ CUtensorMap tmw2, const ConvTcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[8], empty_bar[8], tfull_bar[2], tempty_bar[2];
     __shared__ uint64_t sfull_bar[kMaxOutBufs], sfree_bar[kMaxOutBufs];  // staging buffer: filled by the epilogue / free again (residual landed)
@@ -628,6 +635,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
         tma_prefetch_desc(&tmw);
         if (!POOL) tma_prefetch_desc(&tmy);
         if (!POOL && RES) tma_prefetch_desc(&tmr);
+        if (p.kchunks1 < p.kchunks) { tma_prefetch_desc(&tmx2); tma_prefetch_desc(&tmw2); }
     }
     if (warp == kMmaWarp) {
         tmem_alloc(&tmem_base_s, p.tmem_cols);
@@ -643,7 +651,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap tmx, const __grid_constant__ 
     if (threadIdx.x == 0) DLF_TRACE_POINT(p.status, 1);
     const uint32_t tmem_base = tmem_base_s;
 
-    conv_tc_roles<ACT, POOL, RES, ROW, SPLIT>(&tmx, &tmw, &tmy, &tmr, p, sm, tmem_base, stage0, base, GridSync{nullptr, 0u});
+    conv_tc_roles<ACT, POOL, RES, ROW, SPLIT>(&tmx, &tmw, &tmy, &tmr, &tmx2, &tmw2, p, sm, tmem_base, stage0, base, GridSync{nullptr, 0u});
 
     tc_fence_before_sync();
     __syncthreads();
@@ -682,7 +690,7 @@ struct SeqParams {
 template <int ACT, bool POOL, bool RES, bool ROW>
 __device__ __noinline__ void conv_seq_layer(const SeqLayer* Y, const ConvTcParams* p, const ConvBars* sm, uint32_t tmem_base, uint8_t* stage0,
                                             uint32_t base, unsigned* sync, unsigned target) {
-    conv_tc_roles<ACT, POOL, RES, ROW, false>(&Y->tmx, &Y->tmw, &Y->tmy, &Y->tmr, *p, *sm, tmem_base, stage0, base, GridSync{sync, target});
+    conv_tc_roles<ACT, POOL, RES, ROW, false>(&Y->tmx, &Y->tmw, &Y->tmy, &Y->tmr, &Y->tmx, &Y->tmw, *p, *sm, tmem_base, stage0, base, GridSync{sync, target});
 }
 
 __global__ void __launch_bounds__(kThreads, 1) conv_seq_kernel(const __grid_constant__ SeqParams sp) {
@@ -812,7 +820,8 @@ Tile pick_tile(int N, int Ho, int Wo, int pool) {
     return best;
 }
 
-typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const ConvTcParams);
+typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap,
+                         const ConvTcParams);
 
 template <int ACT, bool POOL, bool RES>
 KernelFn pick_row(bool row) {
@@ -854,10 +863,20 @@ bool conv_tc_supported(const ConvArgs& a) {
     return true;
 }
 
+// The second source joins a 1x1 stride-1 layer chunk by chunk of 64 channels; both channel counts are whole chunks.
+bool conv_tc_dual_supported(const ConvArgs& a) {
+    if (!conv_tc_supported(a)) return false;
+    if (a.kh != 1 || a.kw != 1 || a.stride != 1 || a.pad != 0 || a.pool) return false;
+    if (a.Cin % 64 || a.Cin2 < 64 || a.Cin2 % 64) return false;
+    if (a.stride2 < 1 || a.stride2 > 2) return false;
+    if (a.H2 < 1 || a.W2 < 1 || (a.H2 - 1) / a.stride2 + 1 != a.Ho || (a.W2 - 1) / a.stride2 + 1 != a.Wo) return false;
+    return true;
+}
+
 namespace {
 // Everything a launch of one layer needs: tensor maps, parameters, the kernel variant, shared memory, grid.
 struct ConvTcLaunch {
-    CUtensorMap tmx, tmw, tmy, tmr;
+    CUtensorMap tmx, tmw, tmy, tmr, tmx2, tmw2;
     ConvTcParams p;
     int act, pool, res, row, split;
     size_t smem;
@@ -866,12 +885,14 @@ struct ConvTcLaunch {
 
 int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcLaunch* out) {
     if (!conv_tc_supported(a_in)) return DLF_E_UNSUPPORTED;
+    const bool dual = a_in.x2 != nullptr;
+    if (dual && !conv_tc_dual_supported(a_in)) return DLF_E_UNSUPPORTED;
     // A 1x1 stride-1 convolution has no spatial structure: its N x H x W pixels are one list, cut into tiles of any
     // length, so that the persistent grid's rounds can be filled evenly (below) whatever the image size.
     ConvArgs a = a_in;
     const long long flat_pixels = static_cast<long long>(a_in.N) * a_in.H * a_in.W;
     // (measured to pay for the output-bound layers with few input channels; with more, the image-shaped tiles were as fast or faster)
-    const bool flat = a.kh == 1 && a.kw == 1 && a.stride == 1 && a.pad == 0 && !a.pool && flat_pixels < (1ll << 31) && (a.Cin <= 128 || a.H * a.W == 1);
+    const bool flat = a.kh == 1 && a.kw == 1 && a.stride == 1 && a.pad == 0 && !a.pool && flat_pixels < (1ll << 31) && (a.Cin <= 128 || a.H * a.W == 1) && !dual;
     if (flat) {
         a.N = 1; a.H = 1; a.Ho = 1;
         a.W = a.Wo = static_cast<int>(flat_pixels);
@@ -882,6 +903,11 @@ int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcL
     const int cout16 = (a.Cout + 15) / 16 * 16;
     p.kchunks = (a.Cin + 63) / 64;
     p.ksteps_last = ((a.Cin - (p.kchunks - 1) * 64) + 15) / 16;
+    p.kchunks1 = p.kchunks;
+    if (dual) {   // the second source's chunks follow the first's in K
+        p.kchunks += a.Cin2 / 64;
+        p.stride2 = a.stride2;
+    }
     p.grouped = (a.Cin % 64 == 0) ? 1 : 0;
     Tile tl{};
     long long m_tiles = 0;
@@ -966,7 +992,7 @@ int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcL
     // instruction: max(N / 2, 32 + N / 4) cycles, against 74 bytes per cycle of fill), plus what it writes (and reads as
     // residual) weighted by the ratio of an SM's fill rate to its share of the HBM rate, plus a fixed hand-off cost; sharing
     // a tile costs the fp32 partial tile's round trip and a hand-over on top.  Negative: `sp` shares are not possible.
-    const bool can_split = a.splitk_ws && a.splitk_bytes > kSplitCounterBytes && !a.res && !a.pool;
+    const bool can_split = a.splitk_ws && a.splitk_bytes > kSplitCounterBytes && !a.res && !a.pool && !dual;
     auto split_score = [&](int sp) -> long long {
         const int loads = p.tgroups * p.kgroups;
         const int per = (loads + sp - 1) / sp;
@@ -1079,10 +1105,10 @@ int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcL
     p.acc_stride = (p.BN + 31) / 32 * 32;
     while (cols < static_cast<uint32_t>(2 * p.acc_stride)) cols <<= 1;
     p.tmem_cols = cols;
-    p.bias = a.bias; p.res = static_cast<const __half*>(a.res); p.out = static_cast<__half*>(a.y);
+    p.bias = a.bias; p.bias2 = dual ? a.bias2 : nullptr; p.res = static_cast<const __half*>(a.res); p.out = static_cast<__half*>(a.y);
     p.status = status_dev;
 
-    CUtensorMap tmx, tmw, tmy, tmr;
+    CUtensorMap tmx, tmw, tmy, tmr, tmx2, tmw2;
     const uint64_t taps64 = static_cast<uint64_t>(a.kh) * a.kw;
     if (p.grouped) {
         // input seen as (64 channels, W, H, N, C_in / 64): one box carries one 64-channel chunk of a tap's window
@@ -1119,6 +1145,24 @@ int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcL
         rc = encode_tmap(&tmw, a.w, 3, wdims, wstrides, wbox, wes);
         if (rc) return rc;
     }
+    tmx2 = tmx; tmw2 = tmw;
+    if (dual) {   // the second source, seen like the first: (64 channels, W2, H2, N, Cin2 / 64) read with its own stride
+        const uint64_t dims[5] = {64, static_cast<uint64_t>(a.W2), static_cast<uint64_t>(a.H2), static_cast<uint64_t>(a.N),
+                                  static_cast<uint64_t>(a.Cin2 / 64)};
+        const uint64_t strides[4] = {static_cast<uint64_t>(a.Cin2) * 2, static_cast<uint64_t>(a.W2) * a.Cin2 * 2,
+                                     static_cast<uint64_t>(a.H2) * a.W2 * a.Cin2 * 2, 128};
+        const uint32_t box[5] = {64, static_cast<uint32_t>(tl.tw * a.stride2), static_cast<uint32_t>(tl.th * a.stride2),
+                                 static_cast<uint32_t>(tl.tn), 1};
+        const uint32_t es[5] = {1, static_cast<uint32_t>(a.stride2), static_cast<uint32_t>(a.stride2), 1, 1};
+        int rc = encode_tmap(&tmx2, a.x2, 5, dims, strides, box, es);
+        if (rc) return rc;
+        const uint64_t wdims[4] = {64, static_cast<uint64_t>(a.Cout), 1, static_cast<uint64_t>(a.Cin2 / 64)};
+        const uint64_t wstrides[3] = {static_cast<uint64_t>(a.Cin2) * 2, static_cast<uint64_t>(a.Cin2) * 2, 128};
+        const uint32_t wbox[4] = {64, static_cast<uint32_t>(p.BN), 1, 1};
+        const uint32_t wes[4] = {1, 1, 1, 1};
+        rc = encode_tmap(&tmw2, a.w2, 4, wdims, wstrides, wbox, wes);
+        if (rc) return rc;
+    }
     {   // output map (unused by the pooled variant, which stores from registers)
         const int Hy = a.pool ? a.Ho / 2 : a.Ho, Wy = a.pool ? a.Wo / 2 : a.Wo;
         const uint64_t dims[4] = {static_cast<uint64_t>(a.Cout), static_cast<uint64_t>(Wy), static_cast<uint64_t>(Hy),
@@ -1142,7 +1186,7 @@ int conv_tc_prepare(const ConvArgs& a_in, int sm_count, int* status_dev, ConvTcL
     fprintf(stderr, "conv_tc: tile %dx%dx%d rows %d BN %d x %d splits %d kgs %d kg %d kgroups %d stages %d out_bufs %d work %d grid %d\n", tl.tn, tl.th, tl.tw,
             p.rows, p.BN, p.n_tiles_n, p.splits, p.kgs, p.kg, p.kgroups, p.stages, p.out_bufs, p.n_work, out->grid);
 #endif
-    out->tmx = tmx; out->tmw = tmw; out->tmy = tmy; out->tmr = tmr;
+    out->tmx = tmx; out->tmw = tmw; out->tmy = tmy; out->tmr = tmr; out->tmx2 = tmx2; out->tmw2 = tmw2;
     out->p = p;
     out->act = a.act; out->pool = a.pool != 0; out->res = a.res != nullptr; out->row = p.tps == 3; out->split = splits > 1;
     return DLF_OK;
@@ -1156,7 +1200,7 @@ int launch_conv_tc(const ConvArgs& a, int sm_count, int* status_dev, cudaStream_
     rc = conv_tc_prepare(a, sm_count, status_dev, &L);
     if (rc) return rc;
     const KernelFn fn = L.split ? pick_split(L.act, L.row != 0) : pick_kernel(L.act, L.pool != 0, L.res != 0, L.row != 0);
-    cudaError_t e = launch_kernel(fn, L.grid, kThreads, L.smem, s, L.tmx, L.tmw, L.tmy, L.tmr, L.p);
+    cudaError_t e = launch_kernel(fn, L.grid, kThreads, L.smem, s, L.tmx, L.tmw, L.tmy, L.tmr, L.tmx2, L.tmw2, L.p);
     return e == cudaSuccess ? DLF_OK : cuda_fail(e);
 }
 
@@ -1180,7 +1224,7 @@ int launch_conv_seq(const ConvArgs* layers, int n_layers, int sm_count, int* sta
         ConvTcLaunch L;
         rc = conv_tc_prepare(a, sm_count, status_dev, &L);
         if (rc) return rc;
-        if (L.split || (L.pool && L.row)) return DLF_E_UNSUPPORTED;
+        if (L.split || (L.pool && L.row) || a.x2) return DLF_E_UNSUPPORTED;
         SeqLayer& Y = sp.L[l];
         Y.tmx = L.tmx; Y.tmw = L.tmw; Y.tmy = L.tmy; Y.tmr = L.tmr;
         Y.p = L.p;

@@ -23,7 +23,17 @@ struct ConvArgs {
     // are zero between launches, then room for fp32 partial tiles.  Null: every tile is one work item.
     void* splitk_ws;
     size_t splitk_bytes;
+    // Optional second 1x1 source whose product joins the same accumulator (a residual block's projection branch fused
+    // with its expansion layer): y = act(x * w + bias + x2 * w2 + bias2).  x2 is [N][H2][W2][Cin2], read at
+    // (ho * stride2, wo * stride2); w2 is [Cout][Cin2].  Null x2: an ordinary layer.
+    const void* x2;
+    const void* w2;
+    const float* bias2;
+    int H2, W2, Cin2, stride2;
 };
+
+// True if `a` (with its second source) can run as one conv_tc launch.
+bool conv_tc_dual_supported(const ConvArgs& a);
 
 // A chain of stride-1, size-keeping dense convolutions executed by one kernel.
 constexpr int kMaxChain = 8;

@@ -341,3 +341,20 @@ def test_group_kernel_option_chooses_the_hand_over():
         B.net_set_option(sess.net, B.OPT_GROUP_KERNEL, opt)
         G.check_plan(sess, xd, ref, [2], [sms()], "option %d" % opt)
         assert sess.kernels() == [kernel]
+
+
+# ---- projection branch + expansion layer as one product (K runs over both inputs) ------------------------------------
+@pytest.mark.parametrize("case", [(64, 64, 256, 1, 2, 19, 23), (128, 64, 128, 2, 3, 18, 22), (192, 128, 320, 2, 1, 7, 7),
+                                  (64, 128, 72, 1, 5, 9, 5)])
+def test_projection_and_expansion_as_one_group(case):
+    cin, mid, cout, stride, n, h, w = case
+    layers = [_conv(cin, mid, 1, src=-1), _conv(mid, mid, 3, stride=stride, src=0),
+              _conv(cin, cout, 1, stride=stride, pad=0, act="none", src=-1), _conv(mid, cout, 1, src=1, res_src=2),
+              _conv(cout, 64, 1, src=3)]
+    sess, xd, ref = _mk(layers, "projadd%d" % cin, n, h, w, cin)
+    G.check_plan(sess, xd, ref, [0, 1, 2, 3, 4], [sms()] * 5, "unfused")
+    for s in (sms(), 7, 1):
+        G.check_plan(sess, xd, ref, [0, 1, 3, 4], [sms(), sms(), s, sms()], "projection + expansion S=%d" % s)
+        assert sess.kernels()[2] == "conv_tc"
+    assert B.net_group_is_legal(sess.net, 2, 3, sms())
+    assert B.net_tuner_may_fuse(sess.net, 2, 3, False, sms())
