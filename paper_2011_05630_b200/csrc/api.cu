@@ -179,14 +179,7 @@ static bool depthwise_ok(const dlf_layer_desc& d) {
     return d.op == DLF_DWCONV && d.kh == 3 && d.kw == 3 && d.pad == 1 && (d.stride == 1 || d.stride == 2) && d.pool == 0 &&
            d.res_src == -2;
 }
-// Widest hidden tensor of an inverted-residual block the tuner proposes as one kernel: the kernel walks
-// the hidden channels in 64-wide steps one after the other, and beyond four steps three kernels that
-// each fill the chip were measured faster; so were two kernels for a block without an expansion
-// layer, which the tuner (max_hid > 0) does not propose either.  A plan given explicitly may still ask
-// for both.
-static const int kTunerMaxHidden = 256;
-
-static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix, int max_hid = 0) {
+static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix) {
     const int len = last - first + 1;
     if (len < 2 || len > 3) return false;
     const dlf_layer_desc& d0 = net->layers[first].d;
@@ -210,7 +203,7 @@ static bool span_is_mbconv(const dlf_net* net, int first, int last, bool prefix,
     std::memset(&a, 0, sizeof(a));
     a.N = 1; a.H = 8; a.W = 8;
     a.Cin = has_expand ? d0.cin : hid; a.hid = hid; a.Cout = cout; a.stride = dd.stride; a.has_expand = has_expand ? 1 : 0;
-    if (!mbconv_supported(a) || (max_hid > 0 && (hid > max_hid || !has_expand))) return false;
+    if (!mbconv_supported(a)) return false;
     // the maps between the layers are used nowhere else
     const int n = static_cast<int>(net->layers.size());
     for (int j = first + 1; j < n; j++) {
@@ -486,10 +479,32 @@ static bool chain_pays(const dlf_net* net, int first, int last, int sms, ChainTi
     return t.cost / 1.9e3 + 5.5 < 0.85 * single_us;
 }
 
+// The estimate for an inverted-residual block: the fused kernel's own cost model (the tiler's SM clocks, plus one kernel
+// boundary) against one kernel per layer, each at its bytes at 2.5 TB/s - what the depthwise and the narrow pointwise kernels
+// reach on this chip - plus 5 us of fixed cost; the block must win by a tenth.  It replaces the fixed limit on the hidden
+// width of the first version: wide blocks on small maps (many 64-channel steps, few tiles to spread over the SMs) lose, the
+// same blocks at a large batch win.
+static bool mbconv_pays(const dlf_net* net, int first, int last, int sms) {
+    const MbconvTiling t = mbconv_tiling(mbconv_args(net, first, last, nullptr, nullptr), sms);
+    if (!t.ok) return false;
+    double single_us = 0.0;
+    for (int i = first; i <= last; i++) {
+        const Layer& l = net->layers[i];
+        const double bytes = static_cast<double>(l.in[0] * l.in[1] * l.in[2] * l.in[3] * 2) + static_cast<double>(l.bytes) + static_cast<double>(l.w_elems * 2) +
+                             (l.d.res_src != -2 ? static_cast<double>(l.bytes) : 0.0);
+        single_us += std::max(static_cast<double>(l.flops) / 600e6, bytes / 2.5e6) + 5.0;
+    }
+    return t.cost / 1.9e3 + 5.5 < 0.9 * single_us;
+}
+
 static bool tuner_may_fuse(const dlf_net* net, int first, int last, bool prefix, int s_max) {
     if (first == last) return true;
     if (net->opt_no_tc) return false;
-    if (span_is_mbconv(net, first, last, prefix, kTunerMaxHidden)) return true;
+    if (span_is_mbconv(net, first, last, prefix)) {
+        // (the layers may be the beginning of the block: the estimate is made for the whole of it)
+        const int full_last = first + (net->layers[first].d.op == DLF_CONV ? 2 : 1);
+        return full_last < static_cast<int>(net->layers.size()) && span_is_mbconv(net, first, full_last, false) && mbconv_pays(net, first, full_last, s_max);
+    }
     if (net->opt_group_kernel == 2 && span_is_seq(net, first, last)) return true;
     // a projection and the expansion layer it is added to are one product with a longer K: never slower than the two kernels
     if (span_is_projadd(net, first, last)) return true;

@@ -145,6 +145,7 @@ struct MbconvTiling {
     int out_planes;  // 64-channel planes of the output staging buffer, 0 = none (direct stores)
     size_t smem_bytes;
     double redundancy;
+    double cost;     // the tiler's time estimate (SM clocks)
     bool ok;
 };
 bool mbconv_supported(const MbconvArgs& a);

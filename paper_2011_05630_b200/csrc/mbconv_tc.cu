@@ -773,17 +773,18 @@ MbconvTiling mbconv_tiling(const MbconvArgs& a, int sm_count) {
             const long long n_tiles = static_cast<long long>(a.N) * tiles_h * tiles_w;
             if (n_tiles > 0x7fffffffLL) continue;
             const long long waves = (n_tiles + sm_count - 1) / sm_count;
-            // Per chunk the tensor core issues nbd x 36 depthwise products (N = 16), the expansion and the projection; the
-            // CUDA cores run the two epilogues (a 16-column pass over a 128-row block per warp: about 250 clocks of dependent
-            // instructions, four warps per scheduler).  With both double buffers the two overlap; without, they alternate.
+            // Per chunk (measured cycle accounts of one CTA): the tensor core runs nbd x 9 x (16-channel groups) depthwise
+            // products of 40 clocks, the expansion and the projection; the work warps run the two epilogues, about 500 clocks
+            // of dependent instructions per 128-row block and pass each; the two sides overlap but hand over to each other
+            // four times per chunk (about 1500 clocks of waits).  Without both double buffers they alternate.
             const double jn = std::min(4.0, a.hid / 16.0 / L.chunks);
             const double tc = L.nbd * 9 * jn * 40.0 + (a.has_expand ? L.nb1 * L.kin * 4 * 50.0 : 0.0) + L.nb2 * 4 * std::max(48.0, L.n2 / 2.0);
-            const double cu = (a.has_expand ? 200.0 + 250.0 * L.nb1 : 100.0) + 200.0 + 250.0 * L.nbd;
-            const double overlap = (L.hbufs == 2 && L.ddbufs == 2) ? std::max(tc, cu) + 300.0 : tc + cu;
+            const double cu = (a.has_expand ? 500.0 + 500.0 * L.nb1 : 300.0) + 400.0 + 500.0 * L.nbd;
+            const double per_chunk = (L.hbufs == 2 && L.ddbufs == 2) ? std::max(tc, cu) + 1500.0 : tc + cu + 1000.0;
             // epilogue 2: staged tiles leave by TMA; direct stores touch one cache line per thread and instruction
-            const double epi2 = L.nb2 * (L.n2 / 16.0) * (L.so_planes > 0 ? 80.0 : 320.0);
+            const double epi2 = 1000.0 + L.nb2 * (L.n2 / 16.0) * (L.so_planes > 0 ? 400.0 : 1200.0);
             const double load = L.kin * L.FR * 128 / 64.0;   // the frame through the SM's fill port
-            const double cost = static_cast<double>(waves) * (L.chunks * overlap + epi2 + std::max(0.0, load - L.chunks * overlap) + 2000.0);
+            const double cost = static_cast<double>(waves) * (L.chunks * per_chunk + epi2 + std::max(0.0, load - L.chunks * per_chunk) + 1500.0);
             if (best_cost < 0 || cost < best_cost) {
                 best_cost = cost;
                 best.th = th; best.tw = tw; best.fh = L.fh; best.fw = L.fw; best.nb1 = L.nb1; best.nb2 = L.nb2;
@@ -791,6 +792,7 @@ MbconvTiling mbconv_tiling(const MbconvArgs& a, int sm_count) {
                 best.stages = L.stages; best.stage_bytes = L.stage_bytes;
                 best.smem_bytes = L.smem;
                 best.out_planes = L.so_planes;
+                best.cost = cost;
                 best.redundancy = static_cast<double>(L.FR) / (std::min(th, Ho) * a.stride * std::min(tw, Wo) * a.stride);
                 best.ok = true;
             }
