@@ -134,9 +134,12 @@ int dlf_net_get_plan(const dlf_net* net, int* n_groups, int32_t* group_end, int3
 int dlf_net_group_is_legal(const dlf_net* net, int first, int last, int sm_count);
 
 /* The rule that bounds Algorithm 1's blocks here (the paper's vendor SDK fuses "almost arbitrary" layers, Sec. III-B; this
- * library has three fused kernels): 1 if the tuner may propose layers first..last as one group on s_max SMs - the span is
- * an inverted-residual block up to the measured hidden width, or a dense chain whose fused kernel is estimated (by its own
- * tiler) to beat one kernel per layer, or, with DLF_OPT_GROUP_KERNEL = 2, any run of dense convolutions.  With prefix != 0
+ * library has four fused kernels): 1 if the tuner may propose layers first..last as one group on s_max SMs - the span is
+ * an inverted-residual block or a dense chain whose fused kernel is estimated (by its own tiler) to beat one kernel per
+ * layer, or a residual block's 1x1 projection branch followed by the 1x1 expansion layer it is added to (one product whose
+ * K runs over both inputs: the projection's value joins the fp32 sum without a rounding of its own, at most half an fp16
+ * unit in the last place of that value away from the layer-by-layer result), or, with DLF_OPT_GROUP_KERNEL = 2, any run of
+ * dense convolutions.  With prefix != 0
  * the layers may also be the beginning of an inverted-residual block that can still grow.  0 if not.  Host only. */
 int dlf_net_tuner_may_fuse(const dlf_net* net, int first, int last, int prefix, int s_max);
 

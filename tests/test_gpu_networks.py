@@ -36,6 +36,13 @@ def test_network_every_boundary(name, builder, batch):
     todo = [("unfused", None, None)]
     ends, smc = plans.tuned_plan(sess.net, len(layers))
     todo.append(("tuned", ends, smc))
+    if name == "resnet50":   # the four projection branches run as one product with the expansion layers they are added to
+        assert len(ends) == len(layers) - 4
+        for e in ends:
+            if layers[e]["res_src"] == e - 1:
+                assert e - 1 not in ends
+    if name == "mobilenet_v2":   # inverted-residual blocks run fused where the estimate says the fused kernel pays
+        assert len(ends) < len(layers) - 12
     if name in ("resnet50", "resnet18"):   # one group per residual block (its layers handed over through L2), stem and tail apart
         ends = [0, 1]
         for i in range(2, len(layers) - 2):
