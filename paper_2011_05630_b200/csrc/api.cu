@@ -409,7 +409,13 @@ static bool make_group(const dlf_net* net, int first, int last, int sms, Group* 
     if (first == last) {
         // A single layer runs through the single-layer kernels unless the option asks for the fused-group kernel
         // (a narrow 3x3 layer: 20.5 us in the single-layer kernel's row mode against 26 us here at 56x56x64, batch 32).
-        const bool prefer_chain = net->opt_single_chain != 0;
+        // ... or the layer is a narrow 3x3 layer on an image too wide for the single-layer kernel's row mode (more than 126
+        // pixels): that kernel then re-loads the input window for each of the nine taps, the fused-group kernel loads the
+        // tile's frame once and shifts the operand window (VGG-16's 64 -> 64 layer at 224x224, batch 8: 74.5 -> 52.7 us).
+        const Layer& l1 = net->layers[first];
+        const bool wide_narrow = l1.d.op == DLF_CONV && l1.d.kh == 3 && l1.d.kw == 3 && l1.d.stride == 1 && l1.d.pad == 1 &&
+                                 l1.d.cin <= 64 && l1.d.cout <= 64 && l1.wo_pre + 2 > 128;
+        const bool prefer_chain = net->opt_single_chain != 0 || wide_narrow;
         if (!(prefer_chain && !net->opt_no_tc && span_is_chain(net, first, last))) return single_kind(net, first, &g->kind);
     }
     if (net->opt_no_tc) return false;
