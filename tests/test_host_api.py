@@ -105,7 +105,7 @@ def test_allocation_free_entry_rejects_bad_layers_before_any_launch(layer, statu
 
 
 # ---- the auto-tuner against the restated Algorithm 1 ----------------------------------------------------
-# Which spans one kernel can run, and which of them are worth proposing, is the library's own rule (three fused kernels
+# Which spans one kernel can run, and which of them are worth proposing, is the library's own rule (four fused kernels
 # and their cost estimates - nothing the paper defines): the test takes it from dlf_net_tuner_may_fuse as an INPUT and
 # checks the pass itself - running sums, threshold, deferred close, forced ends, block core count - against oracle/model.py.
 P = dict(alpha=0.316, beta=0.659, kappa=12.0, kappa0=-60.0, s_max=148)
@@ -133,11 +133,18 @@ def test_autotune_equals_restated_algorithm1(name, layers, batch, crit):
                             must_close_after=lambda start, i: i == n - 1 or not can_extend(start, i), may_close=may_close)
     got = B.net_autotune(net, n, P["alpha"], P["beta"], P["kappa"], P["kappa0"], crit, s_max=148, legalise=0)
     assert got == (want[0], want[1]), (got, want)
-    if name == "mobilenet_v2" and crit == 1e30:   # the blocks with a hidden width up to 256 become one group each
+    if name == "mobilenet_v2" and crit == 1e30:   # the blocks whose fused kernel is estimated to pay become one group each
         firsts = [0] + [e + 1 for e in got[0][:-1]]
         assert sum(1 for a, e in zip(firsts, got[0]) if e - a + 1 >= 2) >= 6
     if name == "two_layer" and crit == 1e30:      # the two narrow 3x3 layers: the fused kernel is estimated to pay
         assert got[0] == [1]
+    if name == "resnet50" and crit == 1e30:       # a projection branch and the expansion layer it is added to: one product
+        pairs = [i for i, l in enumerate(layers) if l["res_src"] == i - 1 and l["op"] == "conv"]
+        assert len(pairs) == 4
+        for i in pairs:
+            assert B.net_tuner_may_fuse(net, i - 1, i, False, 148) and i - 1 not in got[0] and i in got[0]
+            assert not B.net_tuner_may_fuse(net, i - 2, i - 1, False, 148)   # (the 3x3 layer does not feed the projection)
+        assert len(got[0]) == n - 4
     B.net_destroy(net)
 
 
